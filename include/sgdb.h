@@ -1,0 +1,244 @@
+/*
+ * sgdb.h -- C ABI of libsgdb: the synchronous parameter-server step with backup
+ * workers ("first N of N+b"), for one NVIDIA B200 (sm_100a).
+ *
+ * Source of the operations: "Revisiting Distributed Synchronous SGD"
+ * (arXiv 1604.00981), Section 3 (backup workers) and Algorithm 4 (Sync-SGD
+ * parameter server): for iteration t the server keeps gradients whose tag equals
+ * t, stops at the N-th such arrival, drops everything else, and updates the
+ * parameters with the mean of the kept N.
+ *
+ * Notation (the paper's): N workers whose gradients are used, b backup workers,
+ * W = N + b rows, t the server's iteration, theta the parameters, G the
+ * gradients.  Workers are numbered 0..W-1 here (the paper counts from 1).
+ *
+ * Conventions shared by every call unless its comment says otherwise
+ *   - `d_` pointers are DEVICE memory and `h_` pointers HOST memory, both owned by
+ *     the caller; the library never frees or keeps them.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls only enqueue work; they never synchronise the stream, except the
+ *     `_host` entry point, which says so.
+ *   - Nothing is allocated by the library; the only memory it touches is what the
+ *     caller passes.
+ *   - Arguments that can be checked on the host (null pointers, N < 1, b < 0,
+ *     N + b > SGDB_MAX_WORKERS, P < 0, ld < P, misaligned base pointers, unknown
+ *     enum values, non-finite hyper-parameters) make the call return
+ *     SGDB_ERR_INVALID_ARG (or SGDB_ERR_UNSUPPORTED) without launching anything.
+ *   - Conditions only the device can see land in a caller-owned device word
+ *     (`d_info`); when that word says SGDB_ERR_INSUFFICIENT, theta, optimizer
+ *     state and mean are left bit-for-bit untouched (Algorithm 4 does not update
+ *     before N current gradients exist).
+ *   - The gradient matrix G is row-major, row w = worker w, `ld` elements between
+ *     row starts (ld >= P), element type sgdb_dtype_t.  theta, optimizer state,
+ *     mean and accumulator are fp32.
+ *   - Base pointers of G, theta, state, mean and acc must be 16-byte aligned in
+ *     the flat calls.  Rows are streamed with 16-byte bulk copies when
+ *     ld * sizeof(element) is a multiple of 16; any other ld is accepted and
+ *     takes an element-wise load path with identical results.
+ *   - Summation order is fixed: the kept rows are added one after another in
+ *     arrival order, starting from +0, in fp32, and the sum is divided by N once.
+ *     Results are therefore bit-reproducible run to run and identical between
+ *     the fused, the separate and the accumulate-on-arrival calls.
+ */
+#ifndef SGDB_H_
+#define SGDB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SGDB_MAX_WORKERS 1024  /* largest accepted W = N + b */
+#define SGDB_MAX_SEGMENTS 4096 /* largest accepted segment-table length */
+
+typedef enum {
+  SGDB_OK = 0,
+  SGDB_ERR_INVALID_ARG = 1,
+  SGDB_ERR_INSUFFICIENT = 2, /* fewer than N workers with tag == t and a finite arrival */
+  SGDB_ERR_CUDA = 3,         /* a CUDA runtime call or a launch failed */
+  SGDB_ERR_UNSUPPORTED = 4,
+  SGDB_ERR_TIMEOUT = 5       /* a bounded on-chip wait ran out (never expected) */
+} sgdb_status_t;
+
+typedef enum { SGDB_F32 = 0, SGDB_BF16 = 1 } sgdb_dtype_t; /* storage type of G's rows */
+
+typedef enum {
+  SGDB_SGD = 0,      /* theta -= lr * g                                   (Section 1.1, SGD rule)      */
+  SGDB_MOMENTUM = 1, /* v = momentum*v + g;  theta -= lr * v                                           */
+  SGDB_RMSPROP = 2,  /* s = decay*s + (1-decay)*g^2;  m = momentum*m + lr*g/sqrt(s+eps);  theta -= m   */
+  SGDB_ADAM = 3      /* m = beta1*m + (1-beta1)*g;  v = beta2*v + (1-beta2)*g^2;
+                        theta -= lr * (m/(1-beta1^step)) / (sqrt(v/(1-beta2^step)) + eps)             */
+} sgdb_opt_kind_t;
+
+/*
+ * Optimizer rule and hyper-parameters, passed by pointer from HOST memory and
+ * read during the call.  g is the mean of the N kept gradients; `lr` multiplies
+ * that mean (Algorithm 4 writes gamma_t / N times the sum).  The paper names the
+ * family (Section 1.1) and uses RMSProp with momentum in its experiments
+ * (Appendix A) without printing equations; the forms above are the ones this
+ * library computes.  state0/state1 per rule: SGD none; MOMENTUM v/-; RMSPROP
+ * s/m; ADAM m/v.  `step` is the 1-based count of updates including this one and
+ * matters to ADAM only.
+ */
+typedef struct sgdb_opt {
+  int32_t kind; /* sgdb_opt_kind_t */
+  float lr;
+  float momentum;
+  float decay;
+  float beta1;
+  float beta2;
+  float eps;
+  int64_t step;
+} sgdb_opt_t;
+
+/*
+ * One tensor of a multi-tensor model (the paper's parameter server updates the
+ * model variable by variable; Section 3.1 follows "one variable", Appendix A.3
+ * sends layers separately).  All pointers are device pointers; only element
+ * alignment (4 bytes, 2 for bf16 gradients) is required, 16-byte alignment of
+ * every pointer and of ld * sizeof(element) selects the fast path per segment.
+ */
+typedef struct sgdb_segment {
+  void *theta;      /* fp32 [len] */
+  void *state0;     /* fp32 [len] or NULL when the rule has no first state  */
+  void *state1;     /* fp32 [len] or NULL when the rule has no second state */
+  const void *grad; /* [W x ld], this tensor's gradient rows, one per worker */
+  int64_t ld;       /* elements between row starts, >= len */
+  int64_t len;      /* elements in this tensor, >= 0 */
+} sgdb_segment_t;
+
+/*
+ * sgdb_select -- which gradients the server uses at iteration t.
+ * Section 3 (the first N to arrive are used, the slowest b are dropped) and
+ * Algorithm 4 (a gradient counts only if its tag equals t).
+ *
+ *   d_arrival [W] fp32   arrival time of worker w's gradient; NaN or +-inf = never arrives
+ *   d_tags    [W] int32  iteration the gradient was computed for
+ *   t, N, b              server iteration, gradients to aggregate, backup workers; W = N + b
+ *   d_mask    [W] uint8  out: 1 for the N kept workers, else 0
+ *   d_order   [N] int32  out: kept worker ids in arrival sequence; equal arrival
+ *                        times are ordered by lower worker id
+ *   d_info    [2] int32  out: {number of valid workers, SGDB_OK or SGDB_ERR_INSUFFICIENT}
+ *
+ * When fewer than N workers are valid, d_mask and d_order are left untouched.
+ */
+sgdb_status_t sgdb_select(const float *d_arrival, const int32_t *d_tags, int32_t t, int32_t N,
+                          int32_t b, uint8_t *d_mask, int32_t *d_order, int32_t *d_info,
+                          void *stream);
+
+/*
+ * sgdb_aggregate -- mean of the kept gradients: (1/N) * sum over the kept G
+ * (the sum in Algorithm 4's update line, before the learning rate).
+ *
+ *   d_grad  [W x ld] rows of type dt;  P columns used;  d_order [N] from sgdb_select
+ *   d_info  [2] or NULL: when given and d_info[1] != SGDB_OK the kernel writes nothing
+ *   d_mean  [P] fp32 out
+ * Rows not named in d_order are never read.
+ */
+sgdb_status_t sgdb_aggregate(const void *d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, int32_t N,
+                             const int32_t *d_order, const int32_t *d_info, float *d_mean,
+                             void *stream);
+
+/*
+ * sgdb_update -- apply the optimizer rule to theta with a given mean gradient
+ * (Algorithm 4's update line; Section 1.1 for the family of rules).
+ *
+ *   d_theta [P] in/out;  d_state0, d_state1 [P] in/out or NULL as the rule needs
+ *   d_mean  [P] in;  opt: host pointer;  d_info as in sgdb_aggregate
+ */
+sgdb_status_t sgdb_update(float *d_theta, float *d_state0, float *d_state1, const float *d_mean,
+                          int64_t P, const sgdb_opt_t *opt, const int32_t *d_info, void *stream);
+
+/*
+ * sgdb_step -- one whole iteration of Algorithm 4's loop body: select,
+ * aggregate and update, with the mean never written to memory.  Arguments as in
+ * the three calls above; d_mask, d_order and d_info are outputs here.
+ */
+sgdb_status_t sgdb_step(const void *d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld,
+                        const float *d_arrival, const int32_t *d_tags, int32_t t, int32_t N,
+                        int32_t b, float *d_theta, float *d_state0, float *d_state1,
+                        const sgdb_opt_t *opt, uint8_t *d_mask, int32_t *d_order, int32_t *d_info,
+                        void *stream);
+
+/*
+ * sgdb_step_segmented -- sgdb_step over a model stored as S separate tensors,
+ * in one launch driven by a table in DEVICE memory (d_segments [S]).  One
+ * selection serves all tensors, as one server iteration does in Algorithm 4.
+ * S <= SGDB_MAX_SEGMENTS, otherwise SGDB_ERR_UNSUPPORTED.
+ */
+sgdb_status_t sgdb_step_segmented(const sgdb_segment_t *d_segments, int32_t S, sgdb_dtype_t dt,
+                                  const float *d_arrival, const int32_t *d_tags, int32_t t,
+                                  int32_t N, int32_t b, const sgdb_opt_t *opt, uint8_t *d_mask,
+                                  int32_t *d_order, int32_t *d_info, void *stream);
+
+/*
+ * sgdb_accumulate_arrival -- Algorithm 4's inner loop taken literally: one
+ * gradient per call, in the order the gradients reach the server.
+ *
+ *   d_row     [P] of type dt   the arriving gradient
+ *   row_tag, t                 its tag and the server's iteration
+ *   d_acc     [P] fp32         running sum, owned by the caller; needs no clearing:
+ *                              the first accepted arrival of an iteration overwrites it
+ *   d_counter [4] int32        server state, zero-initialised once by the caller:
+ *                              {accepted so far, arrivals seen, internal ticket,
+ *                               lowest iteration still open}
+ *   d_info    [2] int32 out    {0 dropped | 1 accumulated | 2 accumulated and updated,
+ *                               accepted count after this call}
+ * A row is accepted iff row_tag == t, t is still open and fewer than N rows have
+ * been accepted; otherwise it is dropped and d_acc is not touched.  The N-th
+ * accepted row triggers mean + optimizer update in the same launch, closes
+ * iteration t and resets the accepted count.  Calls on one stream are ordered by
+ * the stream; there are no device-side waits.  Calls for the same server state
+ * must not overlap on the device.
+ */
+sgdb_status_t sgdb_accumulate_arrival(const void *d_row, sgdb_dtype_t dt, int32_t row_tag,
+                                      int32_t t, int32_t N, int64_t P, float *d_acc,
+                                      int32_t *d_counter, float *d_theta, float *d_state0,
+                                      float *d_state1, const sgdb_opt_t *opt, int32_t *d_info,
+                                      void *stream);
+
+/*
+ * sgdb_step_host -- sgdb_step for a server whose gradients arrive in HOST memory
+ * (the worker-to-server message of Algorithm 3 lands in host buffers) and whose
+ * new parameters go back out to the workers (Algorithm 3 reads theta each
+ * iteration).  theta and the optimizer state stay resident on the device.
+ *
+ *   h_grad [W x ld], h_arrival [W], h_tags [W]   host inputs (pinned memory makes
+ *                                                the copies asynchronous and fast)
+ *   d_theta, d_state0, d_state1                  device, in/out
+ *   h_theta_out [P] or NULL                      host copy of the updated theta
+ *   h_mask [W], h_order [N], h_info [2]          host outputs
+ *   d_workspace, workspace_bytes                 device scratch owned by the caller, at
+ *                                                least sgdb_step_host_workspace_bytes();
+ *                                                16-byte aligned; contents undefined after
+ * Only the N kept rows cross to the device.  The call synchronises `stream`
+ * twice (after selection, and before returning) and returns the device-detected
+ * status, e.g. SGDB_ERR_INSUFFICIENT, directly.
+ */
+sgdb_status_t sgdb_step_host(const void *h_grad, sgdb_dtype_t dt, int64_t P, int64_t ld,
+                             const float *h_arrival, const int32_t *h_tags, int32_t t, int32_t N,
+                             int32_t b, float *d_theta, float *d_state0, float *d_state1,
+                             const sgdb_opt_t *opt, float *h_theta_out, uint8_t *h_mask,
+                             int32_t *h_order, int32_t *h_info, void *d_workspace,
+                             size_t workspace_bytes, void *stream);
+
+/* Bytes of device workspace sgdb_step_host needs for these sizes (0 on invalid sizes). */
+size_t sgdb_step_host_workspace_bytes(sgdb_dtype_t dt, int64_t P, int64_t ld, int32_t N, int32_t b);
+
+/*
+ * sgdb_set_tuning -- launch-shape knobs of the row-streaming kernels, for
+ * measurement sweeps (no counterpart in the paper).  stages: depth of the
+ * shared-memory ring of row slices; ctas_per_sm: resident blocks per SM.
+ * A value <= 0 restores that knob's default.  Affects later calls of this process.
+ */
+sgdb_status_t sgdb_set_tuning(int32_t stages, int32_t ctas_per_sm);
+
+const char *sgdb_strerror(sgdb_status_t status); /* static string, never NULL */
+int sgdb_version(void);                          /* major*10000 + minor*100 + patch */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SGDB_H_ */

@@ -1,0 +1,206 @@
+/*
+ * sgdb_oracle.c -- plain CPU statement of the synchronous parameter-server step
+ * with backup workers, in fp64.
+ *
+ * THIS IS TEST INFRASTRUCTURE.  It exists so that the CUDA library can be checked
+ * against something written straight from the paper.  It is slow on purpose:
+ * single-threaded, one loop per sentence of the method, no blocking, no fusion.
+ * It shares no code, header or table with the CUDA library and neither includes
+ * the other.  Only tests, the smoke check and the CPU-baseline leg of the
+ * benchmark may call it.
+ *
+ * Source: "Revisiting Distributed Synchronous SGD" (arXiv 1604.00981).
+ *   Section 3      -- N + b workers are started; the first N gradients to arrive
+ *                     are used, the slowest b are dropped when they arrive.
+ *   Algorithm 4    -- the server's loop: G = {}; while |G| < N: receive (G, t');
+ *                     keep it iff t' == t; then theta <- theta - gamma_t/N * sum G.
+ *   Section 1.1    -- SGD rule; "update equations differ" for the other rules.
+ *   Appendix A     -- RMSProp with momentum (decay 0.9, momentum 0.9).
+ *
+ * Readings taken where the paper is silent (each also listed in the design notes):
+ *   - two gradients with equal arrival time: the lower worker id arrives first;
+ *   - arrival NaN or +-inf: that gradient never arrives;
+ *   - tag t' > t is dropped like t' < t (Algorithm 4 tests equality);
+ *   - fewer than N current gradients: the server cannot finish the iteration;
+ *     the oracle reports ORACLE_INSUFFICIENT and changes nothing;
+ *   - arrival times are compared as fp32 values, the type they are given in;
+ *   - optimizer equations (the paper prints only SGD's): see oracle_update.
+ *     PARITY UNPINNED BY THE PAPER for momentum / RMSProp / Adam: no equation or
+ *     worked number is printed there; the forms below are pinned by closed forms
+ *     that hold for the chosen reading only.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { ORACLE_OK = 0, ORACLE_INVALID = 1, ORACLE_INSUFFICIENT = 2 };
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+enum { ORACLE_SGD = 0, ORACLE_MOMENTUM = 1, ORACLE_RMSPROP = 2, ORACLE_ADAM = 3 };
+
+typedef struct {
+  int32_t kind;
+  double lr, momentum, decay, beta1, beta2, eps;
+  int64_t step; /* 1-based count of updates, this one included (Adam) */
+} oracle_opt_t;
+
+/* A bf16 value is the upper 16 bits of an fp32 value; widening is exact. */
+static double bf16_bits_to_double(uint16_t bits) {
+  uint32_t u = ((uint32_t)bits) << 16;
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return (double)f;
+}
+
+static double grad_at(const void *grad, int dtype, int64_t index) {
+  if (dtype == ORACLE_BF16) return bf16_bits_to_double(((const uint16_t *)grad)[index]);
+  return (double)((const float *)grad)[index];
+}
+
+/* worker a reaches the server before worker b */
+static int arrives_before(const float *arrival, int32_t a, int32_t b) {
+  if (arrival[a] < arrival[b]) return 1;
+  if (arrival[a] > arrival[b]) return 0;
+  return a < b;
+}
+
+/*
+ * Section 3 + Algorithm 4 (the while loop): the gradients the server ends up
+ * with are the first N to arrive among those tagged t.  Written as its plain
+ * definition: list the valid workers, put them in arrival sequence (insertion
+ * sort), take the first N.
+ *   mask [W]  1 for a kept worker;  order [N] kept ids in arrival sequence;
+ *   n_valid   number of workers with tag == t and a finite arrival time.
+ */
+int oracle_select(const float *arrival, const int32_t *tags, int32_t t, int32_t N, int32_t b,
+                  uint8_t *mask, int32_t *order, int32_t *n_valid) {
+  if (N < 1 || b < 0) return ORACLE_INVALID;
+  int32_t W = N + b;
+  int32_t *seq = (int32_t *)malloc(sizeof(int32_t) * (size_t)W);
+  int32_t count = 0;
+  for (int32_t w = 0; w < W; ++w) {
+    if (tags[w] != t) continue;         /* Algorithm 4: t' == t or the gradient is dropped */
+    if (!isfinite(arrival[w])) continue; /* never arrives */
+    int32_t pos = count++;
+    while (pos > 0 && arrives_before(arrival, w, seq[pos - 1])) {
+      seq[pos] = seq[pos - 1];
+      --pos;
+    }
+    seq[pos] = w;
+  }
+  *n_valid = count;
+  if (count < N) {
+    free(seq);
+    return ORACLE_INSUFFICIENT;
+  }
+  for (int32_t w = 0; w < W; ++w) mask[w] = 0;
+  for (int32_t k = 0; k < N; ++k) { /* the server stops waiting at |G| = N */
+    order[k] = seq[k];
+    mask[seq[k]] = 1;
+  }
+  free(seq);
+  return ORACLE_OK;
+}
+
+/* Algorithm 4's update line, the part before the learning rate: (1/N) sum_{G in set} G. */
+int oracle_aggregate(const void *grad, int dtype, int64_t P, int64_t ld, int32_t N,
+                     const int32_t *order, double *mean) {
+  if (N < 1 || P < 0 || ld < P) return ORACLE_INVALID;
+  for (int64_t i = 0; i < P; ++i) {
+    double sum = 0.0;
+    for (int32_t k = 0; k < N; ++k) sum += grad_at(grad, dtype, (int64_t)order[k] * ld + i);
+    mean[i] = sum / (double)N;
+  }
+  return ORACLE_OK;
+}
+
+/*
+ * The update of theta from the mean gradient g.
+ *   SGD       theta <- theta - lr*g                          (Section 1.1; Algorithm 4 with
+ *                                                             lr = gamma_t, g = sum/N)
+ *   momentum  v <- mu*v + g;  theta <- theta - lr*v
+ *   RMSProp   s <- rho*s + (1-rho)*g^2;  m <- mu*m + lr*g/sqrt(s+eps);  theta <- theta - m
+ *             (Appendix A: "RMSProp with momentum", decay rho, momentum mu)
+ *   Adam      m <- b1*m + (1-b1)*g;  v <- b2*v + (1-b2)*g^2;
+ *             theta <- theta - lr * (m/(1-b1^k)) / (sqrt(v/(1-b2^k)) + eps),  k = step
+ * s0/s1 hold (v,-), (s,m), (m,v) for momentum, RMSProp, Adam.
+ */
+int oracle_update(double *theta, double *s0, double *s1, const double *mean, int64_t P,
+                  const oracle_opt_t *opt) {
+  for (int64_t i = 0; i < P; ++i) {
+    double g = mean[i];
+    switch (opt->kind) {
+      case ORACLE_SGD:
+        theta[i] = theta[i] - opt->lr * g;
+        break;
+      case ORACLE_MOMENTUM:
+        s0[i] = opt->momentum * s0[i] + g;
+        theta[i] = theta[i] - opt->lr * s0[i];
+        break;
+      case ORACLE_RMSPROP:
+        s0[i] = opt->decay * s0[i] + (1.0 - opt->decay) * g * g;
+        s1[i] = opt->momentum * s1[i] + opt->lr * g / sqrt(s0[i] + opt->eps);
+        theta[i] = theta[i] - s1[i];
+        break;
+      case ORACLE_ADAM: {
+        s0[i] = opt->beta1 * s0[i] + (1.0 - opt->beta1) * g;
+        s1[i] = opt->beta2 * s1[i] + (1.0 - opt->beta2) * g * g;
+        double m_hat = s0[i] / (1.0 - pow(opt->beta1, (double)opt->step));
+        double v_hat = s1[i] / (1.0 - pow(opt->beta2, (double)opt->step));
+        theta[i] = theta[i] - opt->lr * m_hat / (sqrt(v_hat) + opt->eps);
+        break;
+      }
+      default:
+        return ORACLE_INVALID;
+    }
+  }
+  return ORACLE_OK;
+}
+
+/* One iteration of Algorithm 4's outer loop: select, aggregate, update. */
+int oracle_step(const void *grad, int dtype, int64_t P, int64_t ld, const float *arrival,
+                const int32_t *tags, int32_t t, int32_t N, int32_t b, double *theta, double *s0,
+                double *s1, const oracle_opt_t *opt, uint8_t *mask, int32_t *order,
+                int32_t *n_valid) {
+  int rc = oracle_select(arrival, tags, t, N, b, mask, order, n_valid);
+  if (rc != ORACLE_OK) return rc;
+  double *mean = (double *)malloc(sizeof(double) * (size_t)(P > 0 ? P : 1));
+  rc = oracle_aggregate(grad, dtype, P, ld, N, order, mean);
+  if (rc == ORACLE_OK) rc = oracle_update(theta, s0, s1, mean, P, opt);
+  free(mean);
+  return rc;
+}
+
+/*
+ * Algorithm 4's while loop, one received gradient per call.
+ *   state[0] = |G| so far, state[1] = gradients received so far,
+ *   state[2] = lowest iteration still open (the server's own t).
+ * Returns through *outcome: 0 dropped, 1 added to the set, 2 added and theta updated.
+ * A gradient is kept iff its tag equals t, iteration t is still open and |G| < N.
+ * On the N-th kept gradient the server updates theta, empties the set and moves
+ * on to t + 1, so anything that still arrives for t is dropped (Section 3).
+ */
+int oracle_accumulate_arrival(const void *row, int dtype, int32_t row_tag, int32_t t, int32_t N,
+                              int64_t P, double *acc, int32_t *state, double *theta, double *s0,
+                              double *s1, const oracle_opt_t *opt, int32_t *outcome) {
+  if (N < 1 || P < 0) return ORACLE_INVALID;
+  state[1] += 1;
+  if (row_tag != t || t < state[2] || state[0] >= N) {
+    *outcome = 0;
+    return ORACLE_OK;
+  }
+  if (state[0] == 0)
+    for (int64_t i = 0; i < P; ++i) acc[i] = 0.0; /* G = {} */
+  for (int64_t i = 0; i < P; ++i) acc[i] += grad_at(row, dtype, i);
+  state[0] += 1;
+  *outcome = 1;
+  if (state[0] == N) {
+    for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)N;
+    int rc = oracle_update(theta, s0, s1, acc, P, opt);
+    if (rc != ORACLE_OK) return rc;
+    state[0] = 0;
+    state[2] = t + 1;
+    *outcome = 2;
+  }
+  return ORACLE_OK;
+}

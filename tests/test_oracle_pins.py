@@ -1,0 +1,398 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked without a GPU.
+
+Each test compares `oracle/` with something that is not the oracle: a hand-worked
+example, a literal replay of Algorithm 4's receive loop, exhaustive enumeration,
+a library routine (numpy mean / argsort, torch's bf16 widening) or a closed form.
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_golden(name):
+    out = {}
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, *vals = line.split()
+            out[key] = vals
+    return out
+
+
+# ---------------------------------------------------------------- hand-worked example
+
+
+def test_hand_worked_iteration():
+    g = _read_golden("alg4_hand_example.txt")
+    t, N, b = int(g["t"][0]), int(g["N"][0]), int(g["b"][0])
+    W = N + b
+    arrival = np.array(g["arrival"], dtype=np.float32)
+    tags = np.array(g["tags"], dtype=np.int32)
+    grad = np.array([g["grad%d" % w] for w in range(W)], dtype=np.float32)
+    theta = np.array(g["theta"], dtype=np.float64)
+    rc, mask, order, n_valid = oracle.select(arrival, tags, t, N, b)
+    assert rc == oracle.OK
+    assert n_valid == int(g["expect_n_valid"][0])
+    assert mask.tolist() == [int(v) for v in g["expect_mask"]]
+    assert order.tolist() == [int(v) for v in g["expect_order"]]
+    mean = oracle.aggregate(grad, 2, order)
+    assert mean.tolist() == [float(v) for v in g["expect_mean"]]
+    rc, mask2, order2, _ = oracle.step(grad, 2, arrival, tags, t, N, b, theta, None, None,
+                                       oracle.Opt(kind=oracle.SGD, lr=float(g["lr"][0])))
+    assert rc == oracle.OK and order2.tolist() == order.tolist() and mask2.tolist() == mask.tolist()
+    assert theta.tolist() == [float(v) for v in g["expect_theta"]]
+
+
+# ---------------------------------------------------------------- selection
+
+
+def _replay_algorithm4(arrival, tags, t, N):
+    """Algorithm 4's loop, event by event: gradients reach the server one at a time in time order
+    (equal times: lower id first); a gradient tagged t joins the set, any other is dropped; the
+    server stops at |set| = N.  Returns the kept ids in the sequence they were received, or None."""
+    W = len(arrival)
+    pending = [w for w in range(W) if math.isfinite(float(arrival[w]))]
+    kept = []
+    while len(kept) < N:
+        if not pending:
+            return None  # the server would wait forever
+        nxt = pending[0]
+        for w in pending[1:]:
+            if float(arrival[w]) < float(arrival[nxt]):  # strict: an equal time keeps the lower id
+                nxt = w
+        pending.remove(nxt)
+        if int(tags[nxt]) == t:
+            kept.append(nxt)
+    return kept
+
+
+def _random_case(rng, W, special=True):
+    values = [0.25, 0.5, 0.5, 1.0, 1.5, 2.0, 7.0]
+    if special:
+        values += [float("inf"), float("nan"), -0.0, 0.0, -1.0, float("-inf")]
+    arrival = np.array([values[i] for i in rng.integers(0, len(values), size=W)], dtype=np.float32)
+    t = int(rng.integers(0, 5))
+    tags = np.where(rng.random(W) < 0.25, t + rng.choice([-1, 1, -2], size=W), t).astype(np.int32)
+    return arrival, tags, t
+
+
+def test_select_matches_replay_of_algorithm4():
+    rng = np.random.default_rng(1)
+    seen_insufficient = seen_ok = 0
+    for trial in range(3000):
+        W = int(rng.integers(1, 9))
+        N = int(rng.integers(1, W + 1))
+        arrival, tags, t = _random_case(rng, W)
+        rc, mask, order, n_valid = oracle.select(arrival, tags, t, N, W - N)
+        kept = _replay_algorithm4(arrival, tags, t, N)
+        valid = [w for w in range(W) if tags[w] == t and math.isfinite(float(arrival[w]))]
+        assert n_valid == len(valid)
+        if kept is None:
+            assert rc == oracle.INSUFFICIENT
+            seen_insufficient += 1
+        else:
+            assert rc == oracle.OK
+            assert order.tolist() == kept
+            assert mask.tolist() == [1 if w in kept else 0 for w in range(W)]
+            seen_ok += 1
+    assert seen_ok > 500 and seen_insufficient > 500
+
+
+def test_select_is_the_unique_earliest_subset():
+    """Enumerate every N-subset of the valid workers: exactly one has all its (time, id) keys below
+    those of every valid worker left out, and it is the oracle's set."""
+    rng = np.random.default_rng(2)
+    for trial in range(400):
+        W = int(rng.integers(2, 9))
+        N = int(rng.integers(1, W + 1))
+        arrival, tags, t = _random_case(rng, W, special=False)
+        valid = [w for w in range(W) if tags[w] == t]
+        rc, mask, order, _ = oracle.select(arrival, tags, t, N, W - N)
+        if len(valid) < N:
+            assert rc == oracle.INSUFFICIENT
+            continue
+        key = lambda w: (float(arrival[w]), w)
+        winners = []
+        for sub in itertools.combinations(valid, N):
+            rest = [w for w in valid if w not in sub]
+            if all(key(a) < key(r) for a in sub for r in rest):
+                winners.append(sub)
+        assert len(winners) == 1
+        assert sorted(order.tolist()) == list(winners[0])
+        assert order.tolist() == sorted(winners[0], key=key)
+
+
+def test_select_special_cases():
+    rng = np.random.default_rng(3)
+    for W in (1, 2, 7, 33, 100, 208, 1024):
+        arrival = rng.lognormal(0, 0.3, size=W).astype(np.float32)
+        arrival[rng.integers(0, W, size=W // 3)] = 1.0  # ties
+        tags = np.full(W, 4, dtype=np.int32)
+        # b = 0, every tag current: all workers kept, in stable argsort order (library routine)
+        rc, mask, order, n_valid = oracle.select(arrival, tags, 4, W, 0)
+        assert rc == oracle.OK and n_valid == W and mask.all()
+        assert order.tolist() == np.argsort(arrival, kind="stable").tolist()
+        # N = 1: the single earliest valid gradient
+        tags2 = tags.copy()
+        tags2[np.argmin(arrival)] = 3  # the earliest one is stale
+        rc, mask, order, _ = oracle.select(arrival, tags2, 4, 1, W - 1)
+        if W == 1:
+            assert rc == oracle.INSUFFICIENT
+            continue
+        cand = np.where(tags2 == 4)[0]
+        best = cand[np.argmin(arrival[cand])]  # argmin returns the first (lowest id) minimum
+        assert rc == oracle.OK and order.tolist() == [best] and mask.sum() == 1 and mask[best] == 1
+
+
+def test_signed_zero_ties_and_never_arriving():
+    arrival = np.array([0.0, -0.0, np.inf, np.nan, -np.inf, -3.0], dtype=np.float32)
+    tags = np.zeros(6, dtype=np.int32)
+    rc, mask, order, n_valid = oracle.select(arrival, tags, 0, 3, 3)
+    assert rc == oracle.OK and n_valid == 3
+    assert order.tolist() == [5, 0, 1]  # -3 first, then +0 and -0 compare equal: lower id first
+    rc, *_ = oracle.select(arrival, tags, 0, 4, 2)
+    assert rc == oracle.INSUFFICIENT
+
+
+def test_stale_tag_removes_worker_and_admits_next():
+    rng = np.random.default_rng(4)
+    W, N, t = 12, 8, 3
+    arrival = rng.permutation(W).astype(np.float32)
+    tags = np.full(W, t, dtype=np.int32)
+    _, mask, order, _ = oracle.select(arrival, tags, t, N, W - N)
+    by_time = np.argsort(arrival, kind="stable").tolist()
+    assert order.tolist() == by_time[:N]
+    victim = order[2]
+    for other in (t - 1, t + 1):  # a tag from the future is dropped like a stale one
+        tags2 = tags.copy()
+        tags2[victim] = other
+        _, mask2, order2, n_valid = oracle.select(arrival, tags2, t, N, W - N)
+        assert n_valid == W - 1 and mask2[victim] == 0
+        assert order2.tolist() == [w for w in by_time if w != victim][:N]
+    rc, mask3, order3, _ = oracle.select(arrival, np.full(W, t - 1, np.int32), t, N, W - N)
+    assert rc == oracle.INSUFFICIENT and not mask3.any() and (order3 == -1).all()  # outputs untouched
+
+
+# ---------------------------------------------------------------- aggregation
+
+
+def test_b0_is_plain_minibatch_mean():
+    """Section 3: with no backups the server averages every worker's gradient."""
+    rng = np.random.default_rng(5)
+    W, P = 17, 1003
+    grad = rng.normal(size=(W, P)).astype(np.float32)
+    arrival = rng.random(W).astype(np.float32)
+    tags = np.zeros(W, np.int32)
+    _, _, order, _ = oracle.select(arrival, tags, 0, W, 0)
+    mean = oracle.aggregate(grad, P, order)
+    ref = grad.astype(np.float64).mean(axis=0)
+    np.testing.assert_allclose(mean, ref, rtol=0, atol=1e-15)
+
+
+def test_constant_rows_give_mean_of_kept_constants():
+    """Divisor is N (not N+b, not the number that arrived) and only kept rows count."""
+    W, N, P = 9, 6, 50
+    consts = np.array([1, 2, 4, 8, 16, 32, 64, 128, 256], dtype=np.float32)  # every subset has its own sum
+    grad = np.repeat(consts[:, None], P, axis=1)
+    arrival = np.array([5, 1, 9, 2, 8, 3, 7, 4, 6], dtype=np.float32)
+    tags = np.array([0, 0, 0, 0, 0, -1, 0, 0, 0], dtype=np.int32)  # worker 5 is stale
+    rc, mask, order, _ = oracle.select(arrival, tags, 0, N, W - N)
+    assert order.tolist() == [1, 3, 7, 0, 8, 6]
+    mean = oracle.aggregate(grad, P, order)
+    expect = (2 + 8 + 128 + 1 + 256 + 64) / 6.0
+    assert (mean == expect).all()
+
+
+def test_leading_dimension_and_column_window():
+    rng = np.random.default_rng(6)
+    W, P, ld = 5, 37, 64
+    grad = rng.normal(size=(W, ld)).astype(np.float32)
+    order = np.array([3, 0, 4], dtype=np.int32)
+    mean = oracle.aggregate(grad, P, order, ld=ld)
+    ref = grad[[3, 0, 4], :P].astype(np.float64).mean(axis=0)
+    np.testing.assert_allclose(mean, ref, rtol=0, atol=1e-15)
+
+
+def test_bf16_widening_matches_torch_for_every_bit_pattern():
+    bits = np.arange(65536, dtype=np.uint16).reshape(1, -1)
+    mean = oracle.aggregate(bits, 65536, np.array([0], dtype=np.int32))
+    ref = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()[0]
+    same = (mean == ref) | (np.isnan(mean) & np.isnan(ref))
+    assert same.all()
+    nonzero = ~np.isnan(ref) & (ref != 0)  # the sum starts from +0, so -0 comes out as +0
+    assert (np.signbit(mean) == np.signbit(ref))[nonzero].all()
+
+
+def _poisoned_copy(grad, mask, rng, value):
+    g = grad.copy()
+    for w in np.where(mask == 0)[0]:
+        g[w] = value if value is not None else rng.normal(size=g.shape[1]) * 1e6
+    return g
+
+
+@pytest.mark.parametrize("kind", [oracle.SGD, oracle.RMSPROP])
+def test_dropped_rows_cannot_influence_theta(kind):
+    """Section 3: late gradients are dropped when they arrive; Algorithm 4: so are wrongly tagged ones."""
+    rng = np.random.default_rng(7)
+    W, N, P, t = 10, 7, 200, 2
+    grad = rng.normal(size=(W, P)).astype(np.float32)
+    arrival = rng.random(W).astype(np.float32)
+    tags = np.full(W, t, np.int32)
+    tags[int(np.argmin(arrival))] = t - 1  # the earliest arrival is stale
+    opt = oracle.Opt(kind=kind, lr=0.05, decay=0.9, momentum=0.9, eps=1.0)
+    results = []
+    for value in ("clean", None, np.nan, np.inf):
+        th = np.linspace(-1, 1, P)
+        s0, s1 = np.zeros(P), np.zeros(P)
+        g = grad if value == "clean" else _poisoned_copy(grad, results[0][3], rng, value)
+        rc, mask, order, _ = oracle.step(g, P, arrival, tags, t, N, W - N, th, s0, s1, opt)
+        assert rc == oracle.OK and mask.sum() == N
+        results.append((th, s0, s1, mask))
+    for th, s0, s1, _ in results[1:]:
+        assert th.tobytes() == results[0][0].tobytes()
+        assert s0.tobytes() == results[0][1].tobytes() and s1.tobytes() == results[0][2].tobytes()
+
+
+def test_insufficient_leaves_everything_untouched():
+    W, N, P = 4, 3, 10
+    grad = np.ones((W, P), np.float32)
+    arrival = np.array([1, 2, np.inf, 3], np.float32)
+    tags = np.array([0, 0, 0, 1], np.int32)
+    th = np.arange(P, dtype=np.float64)
+    s0 = np.full(P, 0.5)
+    rc, mask, order, n_valid = oracle.step(grad, P, arrival, tags, 0, N, 1, th, s0, None,
+                                           oracle.Opt(kind=oracle.MOMENTUM, lr=1.0, momentum=0.5))
+    assert rc == oracle.INSUFFICIENT and n_valid == 2
+    assert (th == np.arange(P)).all() and (s0 == 0.5).all()
+
+
+# ---------------------------------------------------------------- optimizer rules (closed forms)
+
+
+def _run_constant(kind, g, k, theta0=1.5, **hyper):
+    P = len(g)
+    th, s0, s1 = np.full(P, theta0), np.zeros(P), np.zeros(P)
+    out = []
+    for step in range(1, k + 1):
+        oracle.update(th, s0, s1, g, oracle.Opt(kind=kind, step=step, **hyper))
+        out.append(th.copy())
+    return out
+
+
+G_CONST = np.array([-3.0, -0.25, 0.0, 0.5, 2.0, 1e-3])
+
+
+def test_sgd_multi_step_closed_form():
+    """theta_T = theta_0 - lr * sum_t mean_t (Section 1.1), with selection and means from numpy."""
+    rng = np.random.default_rng(8)
+    W, N, P, T, lr = 6, 5, 300, 20, 0.1
+    th = rng.normal(size=P)
+    th0 = th.copy()
+    total = np.zeros(P)
+    for t in range(T):
+        grad = rng.normal(size=(W, P)).astype(np.float32)
+        arrival = rng.lognormal(0, 0.3, W).astype(np.float32)
+        tags = np.full(W, t, np.int32)
+        tags[rng.integers(0, W)] = t - 1
+        rc, *_ = oracle.step(grad, P, arrival, tags, t, N, W - N, th, None, None, oracle.Opt(kind=oracle.SGD, lr=lr))
+        assert rc == oracle.OK
+        kept = _replay_algorithm4(arrival, tags, t, N)
+        total += grad[kept].astype(np.float64).sum(axis=0) / N
+    np.testing.assert_allclose(th, th0 - lr * total, rtol=0, atol=1e-12)
+
+
+def test_momentum_closed_form():
+    mu, lr, k = 0.9, 0.01, 12
+    traj = _run_constant(oracle.MOMENTUM, G_CONST, k, lr=lr, momentum=mu)
+    for j in range(1, k + 1):
+        coeff = sum((1 - mu ** i) / (1 - mu) for i in range(1, j + 1))  # v_i = g (1-mu^i)/(1-mu)
+        np.testing.assert_allclose(traj[j - 1], 1.5 - lr * G_CONST * coeff, rtol=1e-13, atol=1e-15)
+
+
+def test_rmsprop_closed_form():
+    rho, mu, lr, eps, k = 0.9, 0.9, 0.045, 1.0, 6
+    traj = _run_constant(oracle.RMSPROP, G_CONST, k, lr=lr, decay=rho, momentum=mu, eps=eps)
+    # first step from zero state: theta_1 = theta_0 - lr g / sqrt((1-rho) g^2 + eps)
+    np.testing.assert_allclose(traj[0], 1.5 - lr * G_CONST / np.sqrt((1 - rho) * G_CONST ** 2 + eps), rtol=1e-14)
+    # constant g: s_j = (1 - rho^j) g^2 ; m_j = sum_i mu^(j-i) lr g / sqrt(s_i + eps)
+    theta = np.full_like(G_CONST, 1.5)
+    for j in range(1, k + 1):
+        m_j = sum(mu ** (j - i) * lr * G_CONST / np.sqrt((1 - rho ** i) * G_CONST ** 2 + eps) for i in range(1, j + 1))
+        theta = theta - m_j
+        np.testing.assert_allclose(traj[j - 1], theta, rtol=1e-13, atol=1e-15)
+
+
+def test_rmsprop_eps_is_inside_the_root_and_state_is_callers():
+    g = np.array([2.0])
+    th, s, m = np.array([0.0]), np.array([1.0]), np.array([0.5])  # s_0 = 1, m_0 = 0.5
+    oracle.update(th, s, m, g, oracle.Opt(kind=oracle.RMSPROP, lr=1.0, decay=0.5, momentum=0.5, eps=6.5))
+    assert s[0] == 0.5 * 1.0 + 0.5 * 4.0  # 2.5
+    assert m[0] == 0.25 + 2.0 / 3.0  # sqrt(2.5 + 6.5) = 3 ; outside the root it would be sqrt(2.5)+6.5
+    assert th[0] == -m[0]
+
+
+def test_adam_closed_form_every_step():
+    lr, eps, k = 1e-3, 1e-8, 9
+    traj = _run_constant(oracle.ADAM, G_CONST, k, lr=lr, beta1=0.9, beta2=0.999, eps=eps)
+    for j in range(1, k + 1):  # bias-corrected moments equal g and g^2 at every step
+        np.testing.assert_allclose(traj[j - 1], 1.5 - j * lr * G_CONST / (np.abs(G_CONST) + eps), rtol=1e-12, atol=1e-15)
+
+
+def test_adam_eps_is_outside_the_root():
+    g = np.array([3.0])
+    th, m, v = np.array([0.0]), np.array([0.0]), np.array([0.0])
+    oracle.update(th, m, v, g, oracle.Opt(kind=oracle.ADAM, lr=1.0, beta1=0.5, beta2=0.5, eps=1.0, step=1))
+    assert th[0] == pytest.approx(-3.0 / (3.0 + 1.0), rel=1e-15)  # inside the root: -3/sqrt(10)
+
+
+# ---------------------------------------------------------------- arrival-by-arrival server
+
+
+@pytest.mark.parametrize("kind,dtype", [(oracle.SGD, "f32"), (oracle.RMSPROP, "f32"), (oracle.ADAM, "bf16")])
+def test_accumulate_on_arrival_equals_batched(kind, dtype):
+    rng = np.random.default_rng(9)
+    W, N, P, T = 9, 6, 120, 4
+    opt_kw = dict(lr=0.05, decay=0.9, momentum=0.9, beta1=0.9, beta2=0.999, eps=0.1)
+    th_a, s0_a, s1_a = rng.normal(size=P), np.zeros(P), np.zeros(P)
+    th_b, s0_b, s1_b = th_a.copy(), np.zeros(P), np.zeros(P)
+    acc, state = np.full(P, np.nan), oracle.new_server_state()  # acc needs no clearing by the caller
+    leftovers = []  # (row, tag) that arrive after their iteration closed
+    for t in range(T):
+        grad = rng.normal(size=(W, P)).astype(np.float32)
+        if dtype == "bf16":
+            grad = torch.from_numpy(grad).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        arrival = rng.lognormal(0, 0.3, W).astype(np.float32)
+        arrival[2] = arrival[5]  # a tie
+        tags = np.full(W, t, np.int32)
+        tags[int(rng.integers(0, W))] = t - 1
+        opt = oracle.Opt(kind=kind, step=t + 1, **opt_kw)
+        rc, mask, order, _ = oracle.step(grad, P, arrival, tags, t, N, W - N, th_b, s0_b, s1_b, opt)
+        assert rc == oracle.OK
+        outcomes = {}
+        for row, tag in leftovers:  # stragglers of t-1 reach the server during t: dropped
+            assert oracle.accumulate_arrival(row, tag, t, N, acc, state, th_a, s0_a, s1_a, opt) == 0
+        leftovers = []
+        fired = False
+        for w in np.argsort(arrival, kind="stable"):
+            res = oracle.accumulate_arrival(grad[w], int(tags[w]), t, N, acc, state, th_a, s0_a, s1_a, opt)
+            outcomes[int(w)] = res
+            if fired:
+                assert res == 0  # Section 3: the slowest b are dropped when they arrive
+            fired = fired or res == 2
+        assert fired
+        assert [w for w in np.argsort(arrival, kind="stable") if outcomes[int(w)] > 0] == order.tolist()
+        assert state[0] == 0 and state[2] == t + 1
+        np.testing.assert_allclose(th_a, th_b, rtol=1e-13, atol=1e-14)
+        np.testing.assert_allclose(s0_a, s0_b, rtol=1e-13, atol=1e-14)
+        np.testing.assert_allclose(s1_a, s1_b, rtol=1e-13, atol=1e-14)
+        leftovers = [(grad[w], int(tags[w])) for w in range(W) if mask[w] == 0 and tags[w] == t][:1]
