@@ -1,0 +1,327 @@
+#!/usr/bin/env python
+"""Benchmark of the fused N-of-(N+b) aggregate + update step (sgdb_step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl native|reference]
+
+A step is one pass of the whole path over one batch of synthetic input: select the first N of the
+N+b gradients, average them, apply RMSProp with momentum.  The workload is the Inception-v3-sized
+one: P = 23.8 M fp32 parameters, W = 100 (N = 96, b = 4).  Prints one JSON line.
+
+value     gradient bytes read per second (N * P * 4 per step), inputs resident in HBM
+e2e       the same metric through sgdb_step_host: gradients, arrival times and tags start in pinned
+          host memory, the updated parameters are read back, all inside the timed region
+roofline  algorithmic bytes of a step (gradient rows + parameters and state read and written) over
+          the measured step time, against the measured HBM copy bandwidth of this machine
+With --gpus N > 1 (under torchrun) every rank is one parameter-server shard holding its own P
+columns; there is no data-path collective, and the value is the sum over ranks over the slowest rank.
+--impl reference times the CPU oracle on a bounded column sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_1604_00981_b200 import workload as wl
+
+METRIC = "N-of-(N+b) aggregate+update: gradient GB/s read"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0  # earlier measurement on this machine, used only when MEASURED_PEAKS.json is absent
+NOMINAL_HBM_GBS = 8000.0
+
+# DRAM traffic of one fused-step launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
+# as bytes per algorithmic byte; valid only for the kernel sources whose digest is recorded with it.
+NCU_TRAFFIC = {"src_digest": None, "dram_bytes_per_algorithmic_byte": None}
+
+
+def kernel_source_digest() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_1604_00981_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_sample_run(cfg, P_sample: int, steps: int, warmup: int, seed_shift: int = 0):
+    """Times the CPU oracle, as it stands, on the first P_sample columns of the workload.
+    Returns (seconds per step, gradient GB/s)."""
+    import oracle
+
+    W, N = cfg.W, cfg.N
+    scales = wl.worker_scales(cfg.seed, W)
+    grad = wl.as_oracle_array(wl.grad_matrix(cfg.seed + seed_shift, 0, W, P_sample, scales, cfg.grad_dtype, "cpu"))
+    theta = wl.theta0(cfg.seed, P_sample, "cpu").numpy().astype(np.float64)
+    s0, s1 = np.zeros(P_sample), np.zeros(P_sample)
+    hyper = {k: float(np.float32(v)) for k, v in cfg.opt.items() if k != "kind"}
+    kind = {"sgd": oracle.SGD, "momentum": oracle.MOMENTUM, "rmsprop": oracle.RMSPROP, "adam": oracle.ADAM}[cfg.opt["kind"]]
+    times = []
+    for t in range(warmup + steps):
+        arrival, tags = wl.arrivals(cfg.seed, t, W), wl.tags(cfg.seed, t, W, N)
+        t0 = time.perf_counter()
+        rc, *_ = oracle.step(grad, P_sample, arrival, tags, t, N, cfg.b, theta, s0, s1,
+                             oracle.Opt(kind=kind, step=t + 1, **hyper))
+        dt = time.perf_counter() - t0
+        assert rc == oracle.OK
+        if t >= warmup:
+            times.append(dt)
+    sec = float(np.mean(times))
+    esize = 4 if cfg.grad_dtype == "f32" else 2
+    return sec, N * P_sample * esize / sec / 1e9
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    P_sample = cfg.P // 4
+    sec, gbs = oracle_sample_run(cfg, P_sample, args.steps, args.warmup)
+    sample = "first %d of %d columns (1/4), all %d rows, %d steps, single thread" % (P_sample, cfg.P, cfg.W, args.steps)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "P": cfg.P, "W": cfg.W, "N": cfg.N, "b": cfg.b, "optimizer": cfg.opt["kind"],
+                   "grad_dtype": cfg.grad_dtype, "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_native(args, cfg):
+    from paper_1604_00981_b200 import binding as sgdb
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
+    seed = cfg.seed + 1000 * rank  # every rank is its own parameter-server shard
+    scales = wl.worker_scales(cfg.seed, W)
+    grad = wl.grad_matrix(seed, 0, W, P, scales, cfg.grad_dtype, dev)
+    theta = wl.theta0(seed, P, dev)
+    s0 = torch.zeros(P, device=dev)
+    s1 = torch.zeros(P, device=dev)
+    mask = torch.zeros(W, dtype=torch.uint8, device=dev)
+    order = torch.zeros(N, dtype=torch.int32, device=dev)
+    info = torch.zeros(2, dtype=torch.int32, device=dev)
+    n_sets = 16  # arrival/tag draws rotate, so the kept set differs from step to step
+    arr_d = [torch.from_numpy(wl.arrivals(cfg.seed, t, W)).to(dev) for t in range(n_sets)]
+    tag_d = [torch.from_numpy(wl.tags(cfg.seed, t, W, N) - t).to(dev) for t in range(n_sets)]  # tags relative to t = 0
+    opt = sgdb.Opt(**cfg.opt)
+    esize = grad.element_size()
+    grad_bytes = N * P * esize
+    n_state = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2}[cfg.opt["kind"]]
+    total_bytes = grad_bytes + 2 * (1 + n_state) * P * 4
+
+    def step(i):
+        opt.step = i + 1
+        sgdb.sgdb_step(grad, P, arr_d[i % n_sets], tag_d[i % n_sets], 0, N, b, theta, s0, s1, opt, mask, order, info)
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        start.record()
+        for i in range(args.steps):
+            step(args.warmup + i)
+        stop.record()
+        barrier()
+    ms_total = start.elapsed_time(stop)
+    assert info.cpu().tolist()[1] == 0, "a step reported a device-side error"
+    assert bool(torch.isfinite(theta).all())
+
+    # ---- end to end: gradients start in pinned host memory, new parameters are read back
+    e2e_steps = max(1, min(args.steps, 3))
+    ws = torch.empty(sgdb.sgdb_step_host_workspace_bytes(grad.dtype, P, P, N, b), dtype=torch.uint8, device=dev)
+    h_grad = torch.empty((W, P), dtype=grad.dtype, pin_memory=True)
+    h_grad.copy_(grad)
+    del grad
+    h_theta = torch.empty(P, dtype=torch.float32, pin_memory=True)
+    h_mask = torch.empty(W, dtype=torch.uint8, pin_memory=True)
+    h_order = torch.empty(N, dtype=torch.int32, pin_memory=True)
+    h_info = torch.empty(2, dtype=torch.int32, pin_memory=True)
+    h_arr = [torch.from_numpy(wl.arrivals(cfg.seed, t, W)).pin_memory() for t in range(n_sets)]
+    h_tag = [torch.from_numpy(wl.tags(cfg.seed, t, W, N) - t).pin_memory() for t in range(n_sets)]
+
+    def host_step(i):
+        opt.step = i + 1
+        st = sgdb.sgdb_step_host(h_grad, P, h_arr[i % n_sets], h_tag[i % n_sets], 0, N, b, theta, s0, s1, opt,
+                                 h_theta, h_mask, h_order, h_info, ws)
+        assert st == 0
+
+    host_step(0)
+    barrier()
+    e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e_start.record()
+    for i in range(e2e_steps):
+        host_step(1 + i)
+    e_stop.record()
+    barrier()
+    e2e_ms = e_start.elapsed_time(e_stop)
+
+    # ---- max over ranks
+    if dist is not None:
+        tt = torch.tensor([ms_total, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total, e2e_ms = float(tt[0]), float(tt[1])
+    ms_per_step = ms_total / args.steps
+    value = world * grad_bytes / (ms_per_step * 1e-3) / 1e9
+    total_gbs_per_gpu = total_bytes / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * grad_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9
+
+    if rank == 0:
+        peak, peak_kind = measured_hbm_peak()
+        digest = kernel_source_digest()
+        traffic = None
+        if NCU_TRAFFIC["src_digest"] == digest and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] is not None:
+            traffic = NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] * total_bytes
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            P_sample = P // 4
+            sec, gbs = oracle_sample_run(cfg, P_sample, steps=10, warmup=1)
+            cpu = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
+                   "sample": "first %d of %d columns (1/4), all %d rows, 10 steps of %.2f s, single thread"
+                             % (P_sample, P, W, sec)}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": cfg.name, "P": P, "W": W, "N": N, "b": b, "optimizer": cfg.opt["kind"],
+                       "grad_dtype": cfg.grad_dtype, "sharding": "one parameter-server column shard of P per GPU",
+                       "l2": "inputs larger than L2: %.2f GB of gradient rows and %.0f MB of parameters and state per step"
+                             % (grad_bytes / 1e9, (total_bytes - grad_bytes) / 2e6)},
+            "step_us": ms_per_step * 1e3,
+            "total_gbs_per_gpu": total_gbs_per_gpu,
+            "pct_of_nominal_8tbs": 100.0 * total_gbs_per_gpu / NOMINAL_HBM_GBS,
+            "roofline": {"bound": "hbm", "achieved": total_gbs_per_gpu, "peak": peak, "unit": "GB/s",
+                         "frac": total_gbs_per_gpu / peak, "traffic": traffic, "peak_source": peak_kind,
+                         "kernel": "stream_rows_kernel<float, rmsprop> (duration = whole step, including the one-warp select launch)",
+                         "algorithmic_bytes_per_launch": total_bytes},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": N * P * esize + W * 8,
+                    "d2h_bytes_per_step": P * 4 + W + N * 4 + 16, "steps": e2e_steps,
+                    "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": 2 * args.steps,
+            "clocks": clocks.summary(),
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["native", "reference"], default="native")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "native":
+        args.warmup = 3
+    cfg = wl.CONFIGS[1]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_native(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,477 @@
+// Host side of libsgdb: argument checks, launch shapes and the C ABI declared in
+// include/sgdb.h.  Nothing here allocates device memory, and no call synchronises
+// the stream except sgdb_step_host, whose results are host buffers.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+
+#include "sgdb_kernels.cuh"
+
+namespace {
+
+using namespace sgdb;
+
+constexpr int kVersion = 100;  // 0.1.0
+constexpr int kMaxDevices = 64;
+
+// Launch shape of the row-streaming kernel: 256 consumer threads + one producer warp,
+// CH 16-byte chunks per thread and row, so a ring slot holds 8 KiB (f32) / 8 KiB (bf16).
+constexpr int kNT = 256;
+constexpr int kCH = 2;
+constexpr int kStageBytes = kNT * kCH * 16;
+constexpr int kDefaultStages = 12;
+constexpr int kDefaultCtasPerSm = 2;
+
+struct DeviceInfo {
+  bool known = false;
+  int sms = 0;
+  int max_smem_optin = 0;
+};
+DeviceInfo g_dev[kMaxDevices];
+int g_stages = kDefaultStages;
+int g_ctas_per_sm = kDefaultCtasPerSm;
+
+bool is_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+sgdb_status_t device_info(const DeviceInfo** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SGDB_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return SGDB_ERR_UNSUPPORTED;
+  DeviceInfo& d = g_dev[dev];
+  if (!d.known) {
+    if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) !=
+            cudaSuccess)
+      return SGDB_ERR_CUDA;
+    d.known = true;
+  }
+  *out = &d;
+  return SGDB_OK;
+}
+
+sgdb_status_t launch_status() {
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    std::fprintf(stderr, "libsgdb: CUDA error: %s\n", cudaGetErrorString(e));
+    return SGDB_ERR_CUDA;
+  }
+  return SGDB_OK;
+}
+
+bool dtype_ok(int dt) { return dt == SGDB_F32 || dt == SGDB_BF16; }
+size_t dtype_size(int dt) { return dt == SGDB_BF16 ? 2 : 4; }
+
+// Checks the optimizer description and the state pointers its rule needs; derives
+// the constants the kernels use.  `ep` receives the epilogue selector.
+sgdb_status_t prepare_rule(const sgdb_opt_t* opt, const void* state0, const void* state1, Hyper* h,
+                           int* ep) {
+  if (opt == nullptr) return SGDB_ERR_INVALID_ARG;
+  std::memset(h, 0, sizeof(*h));
+  if (!std::isfinite(opt->lr)) return SGDB_ERR_INVALID_ARG;
+  h->lr = opt->lr;
+  switch (opt->kind) {
+    case SGDB_SGD:
+      *ep = EP_SGD;
+      return SGDB_OK;
+    case SGDB_MOMENTUM:
+      if (!std::isfinite(opt->momentum) || state0 == nullptr) return SGDB_ERR_INVALID_ARG;
+      h->mu = opt->momentum;
+      *ep = EP_MOMENTUM;
+      return SGDB_OK;
+    case SGDB_RMSPROP:
+      if (!std::isfinite(opt->momentum) || !std::isfinite(opt->decay) || !std::isfinite(opt->eps) ||
+          state0 == nullptr || state1 == nullptr)
+        return SGDB_ERR_INVALID_ARG;
+      h->mu = opt->momentum;
+      h->rho = opt->decay;
+      h->one_minus_rho = static_cast<float>(1.0 - static_cast<double>(opt->decay));
+      h->eps = opt->eps;
+      *ep = EP_RMSPROP;
+      return SGDB_OK;
+    case SGDB_ADAM: {
+      if (!std::isfinite(opt->beta1) || !std::isfinite(opt->beta2) || !std::isfinite(opt->eps) ||
+          opt->beta1 < 0.f || opt->beta1 >= 1.f || opt->beta2 < 0.f || opt->beta2 >= 1.f ||
+          opt->step < 1 || state0 == nullptr || state1 == nullptr)
+        return SGDB_ERR_INVALID_ARG;
+      h->b1 = opt->beta1;
+      h->b2 = opt->beta2;
+      h->one_minus_b1 = static_cast<float>(1.0 - static_cast<double>(opt->beta1));
+      h->one_minus_b2 = static_cast<float>(1.0 - static_cast<double>(opt->beta2));
+      h->eps = opt->eps;
+      const double k = static_cast<double>(opt->step);
+      h->bc1 = static_cast<float>(1.0 - std::pow(static_cast<double>(opt->beta1), k));
+      h->bc2 = static_cast<float>(1.0 - std::pow(static_cast<double>(opt->beta2), k));
+      *ep = EP_ADAM;
+      return SGDB_OK;
+    }
+    default:
+      return SGDB_ERR_INVALID_ARG;
+  }
+}
+
+sgdb_status_t check_selection_args(const void* arrival, const void* tags, int32_t N, int32_t b,
+                                   const void* mask, const void* order, const void* info) {
+  if (arrival == nullptr || tags == nullptr || mask == nullptr || order == nullptr || info == nullptr)
+    return SGDB_ERR_INVALID_ARG;
+  if (N < 1 || b < 0) return SGDB_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(N) + b > SGDB_MAX_WORKERS) return SGDB_ERR_INVALID_ARG;
+  return SGDB_OK;
+}
+
+// ---------------------------------------------------------------- row-streaming launch
+
+template <typename GT, int EP>
+sgdb_status_t launch_stream_t(const StreamParams& p_in, long long total_tiles_hint, cudaStream_t stream) {
+  const DeviceInfo* dev = nullptr;
+  sgdb_status_t st = device_info(&dev);
+  if (st != SGDB_OK) return st;
+  StreamParams p = p_in;
+  auto kernel = stream_rows_kernel<GT, EP, kNT, kCH>;
+
+  // shared memory: ring + 2 barriers per slot + order[N] + tile prefix[S + 1]
+  const size_t fixed = static_cast<size_t>((p.N + 3) & ~3) * 4 + (p.table ? (static_cast<size_t>(p.S) + 1) * 4 : 0) + 16;
+  int ctas_per_sm = g_ctas_per_sm;
+  int stages = g_stages;
+  const size_t per_sm_budget = static_cast<size_t>(dev->max_smem_optin);
+  // keep the requested residency: shrink the ring until `ctas_per_sm` blocks fit (1 KiB reserved per block)
+  while (stages > 2 &&
+         (static_cast<size_t>(stages) * (kStageBytes + 16) + fixed + 1024) * ctas_per_sm > per_sm_budget + 1024)
+    --stages;
+  const size_t smem = static_cast<size_t>(stages) * (kStageBytes + 16) + fixed;
+  if (smem > per_sm_budget) return SGDB_ERR_UNSUPPORTED;
+  p.stages = stages;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
+      cudaSuccess)
+    return launch_status();
+  long long grid = static_cast<long long>(dev->sms) * ctas_per_sm;
+  if (total_tiles_hint > 0 && total_tiles_hint < grid) grid = total_tiles_hint;
+  if (grid < 1) grid = 1;
+  kernel<<<static_cast<unsigned>(grid), kNT + 32, smem, stream>>>(p);
+  return launch_status();
+}
+
+template <typename GT>
+sgdb_status_t launch_stream_ep(int ep, const StreamParams& p, long long tiles, cudaStream_t stream) {
+  switch (ep) {
+    case EP_MEAN: return launch_stream_t<GT, EP_MEAN>(p, tiles, stream);
+    case EP_SGD: return launch_stream_t<GT, EP_SGD>(p, tiles, stream);
+    case EP_MOMENTUM: return launch_stream_t<GT, EP_MOMENTUM>(p, tiles, stream);
+    case EP_RMSPROP: return launch_stream_t<GT, EP_RMSPROP>(p, tiles, stream);
+    case EP_ADAM: return launch_stream_t<GT, EP_ADAM>(p, tiles, stream);
+  }
+  return SGDB_ERR_INVALID_ARG;
+}
+
+sgdb_status_t launch_stream(int dt, int ep, const StreamParams& p, long long tiles, cudaStream_t stream) {
+  return dt == SGDB_BF16 ? launch_stream_ep<BF16>(ep, p, tiles, stream)
+                         : launch_stream_ep<float>(ep, p, tiles, stream);
+}
+
+long long tiles_of(int dt, long long len) {
+  const long long tile = static_cast<long long>(kNT) * kCH * (dt == SGDB_BF16 ? 8 : 4);
+  return (len + tile - 1) / tile;
+}
+
+sgdb_status_t launch_select(const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t N, int32_t b,
+                            uint8_t* d_mask, int32_t* d_order, int32_t* d_info, cudaStream_t stream) {
+  select_first_n_kernel<<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, N + b, d_mask, d_order, d_info);
+  return launch_status();
+}
+
+sgdb_status_t check_flat(const void* grad, int dt, int64_t P, int64_t ld, int32_t N) {
+  if (grad == nullptr || !dtype_ok(dt)) return SGDB_ERR_INVALID_ARG;
+  if (P < 0 || ld < P || N < 1 || N > SGDB_MAX_WORKERS) return SGDB_ERR_INVALID_ARG;
+  if (!is_aligned16(grad)) return SGDB_ERR_INVALID_ARG;
+  if (tiles_of(dt, P) > 0x7fffffffLL) return SGDB_ERR_UNSUPPORTED;
+  return SGDB_OK;
+}
+
+}  // namespace
+
+// ====================================================================== C ABI
+
+extern "C" {
+
+sgdb_status_t sgdb_select(const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t N, int32_t b,
+                          uint8_t* d_mask, int32_t* d_order, int32_t* d_info, void* stream) {
+  sgdb_status_t st = check_selection_args(d_arrival, d_tags, N, b, d_mask, d_order, d_info);
+  if (st != SGDB_OK) return st;
+  return launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, static_cast<cudaStream_t>(stream));
+}
+
+sgdb_status_t sgdb_aggregate(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, int32_t N,
+                             const int32_t* d_order, const int32_t* d_info, float* d_mean, void* stream) {
+  sgdb_status_t st = check_flat(d_grad, dt, P, ld, N);
+  if (st != SGDB_OK) return st;
+  if (d_order == nullptr || d_mean == nullptr || !is_aligned16(d_mean)) return SGDB_ERR_INVALID_ARG;
+  if (P == 0) return SGDB_OK;
+  StreamParams p{};
+  p.table = nullptr;
+  p.flat.theta = d_mean;
+  p.flat.grad = d_grad;
+  p.flat.ld = ld;
+  p.flat.len = P;
+  p.S = 1;
+  p.N = N;
+  p.order = d_order;
+  p.info = d_info;
+  p.status_out = nullptr;
+  return launch_stream(dt, EP_MEAN, p, tiles_of(dt, P), static_cast<cudaStream_t>(stream));
+}
+
+sgdb_status_t sgdb_update(float* d_theta, float* d_state0, float* d_state1, const float* d_mean, int64_t P,
+                          const sgdb_opt_t* opt, const int32_t* d_info, void* stream) {
+  Hyper h;
+  int ep = 0;
+  sgdb_status_t st = prepare_rule(opt, d_state0, d_state1, &h, &ep);
+  if (st != SGDB_OK) return st;
+  if (d_theta == nullptr || d_mean == nullptr || P < 0) return SGDB_ERR_INVALID_ARG;
+  if (!is_aligned16(d_theta) || !is_aligned16(d_mean) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
+    return SGDB_ERR_INVALID_ARG;
+  if (P == 0) return SGDB_OK;
+  const DeviceInfo* dev = nullptr;
+  st = device_info(&dev);
+  if (st != SGDB_OK) return st;
+  UpdateParams p{d_theta, d_state0, d_state1, d_mean, P, d_info, h};
+  const long long chunks = (P + 3) / 4;
+  long long grid = (chunks + 255) / 256;
+  const long long cap = static_cast<long long>(dev->sms) * 8;
+  if (grid > cap) grid = cap;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  switch (ep) {
+    case EP_SGD: update_kernel<EP_SGD><<<static_cast<unsigned>(grid), 256, 0, s>>>(p); break;
+    case EP_MOMENTUM: update_kernel<EP_MOMENTUM><<<static_cast<unsigned>(grid), 256, 0, s>>>(p); break;
+    case EP_RMSPROP: update_kernel<EP_RMSPROP><<<static_cast<unsigned>(grid), 256, 0, s>>>(p); break;
+    case EP_ADAM: update_kernel<EP_ADAM><<<static_cast<unsigned>(grid), 256, 0, s>>>(p); break;
+    default: return SGDB_ERR_INVALID_ARG;
+  }
+  return launch_status();
+}
+
+sgdb_status_t sgdb_step(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, const float* d_arrival,
+                        const int32_t* d_tags, int32_t t, int32_t N, int32_t b, float* d_theta,
+                        float* d_state0, float* d_state1, const sgdb_opt_t* opt, uint8_t* d_mask,
+                        int32_t* d_order, int32_t* d_info, void* stream) {
+  sgdb_status_t st = check_selection_args(d_arrival, d_tags, N, b, d_mask, d_order, d_info);
+  if (st != SGDB_OK) return st;
+  st = check_flat(d_grad, dt, P, ld, N);
+  if (st != SGDB_OK) return st;
+  Hyper h;
+  int ep = 0;
+  st = prepare_rule(opt, d_state0, d_state1, &h, &ep);
+  if (st != SGDB_OK) return st;
+  if (d_theta == nullptr || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
+    return SGDB_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
+  if (st != SGDB_OK || P == 0) return st;
+  StreamParams p{};
+  p.table = nullptr;
+  p.flat.theta = d_theta;
+  p.flat.state0 = d_state0;
+  p.flat.state1 = d_state1;
+  p.flat.grad = d_grad;
+  p.flat.ld = ld;
+  p.flat.len = P;
+  p.S = 1;
+  p.N = N;
+  p.order = d_order;
+  p.info = d_info;
+  p.status_out = d_info + 1;
+  p.h = h;
+  return launch_stream(dt, ep, p, tiles_of(dt, P), s);
+}
+
+sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, sgdb_dtype_t dt,
+                                  const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t N,
+                                  int32_t b, const sgdb_opt_t* opt, uint8_t* d_mask, int32_t* d_order,
+                                  int32_t* d_info, void* stream) {
+  sgdb_status_t st = check_selection_args(d_arrival, d_tags, N, b, d_mask, d_order, d_info);
+  if (st != SGDB_OK) return st;
+  if (d_segments == nullptr || S < 0 || !dtype_ok(dt)) return SGDB_ERR_INVALID_ARG;
+  if (S > SGDB_MAX_SEGMENTS) return SGDB_ERR_UNSUPPORTED;
+  Hyper h;
+  int ep = 0;
+  // the table lives on the device; whether each segment carries the state pointers its
+  // rule needs cannot be seen from here, so only the rule itself is checked
+  const int dummy = 0;
+  st = prepare_rule(opt, &dummy, &dummy, &h, &ep);
+  if (st != SGDB_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
+  if (st != SGDB_OK || S == 0) return st;
+  StreamParams p{};
+  p.table = d_segments;
+  p.S = S;
+  p.N = N;
+  p.order = d_order;
+  p.info = d_info;
+  p.status_out = d_info + 1;
+  p.h = h;
+  return launch_stream(dt, ep, p, 0, s);
+}
+
+sgdb_status_t sgdb_accumulate_arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag, int32_t t,
+                                      int32_t N, int64_t P, float* d_acc, int32_t* d_counter,
+                                      float* d_theta, float* d_state0, float* d_state1,
+                                      const sgdb_opt_t* opt, int32_t* d_info, void* stream) {
+  if (d_row == nullptr || d_acc == nullptr || d_counter == nullptr || d_theta == nullptr || d_info == nullptr)
+    return SGDB_ERR_INVALID_ARG;
+  if (!dtype_ok(dt) || N < 1 || P < 0) return SGDB_ERR_INVALID_ARG;
+  if (!is_aligned16(d_acc) || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1) ||
+      !is_aligned16(d_row))
+    return SGDB_ERR_INVALID_ARG;
+  Hyper h;
+  int ep = 0;
+  sgdb_status_t st = prepare_rule(opt, d_state0, d_state1, &h, &ep);
+  if (st != SGDB_OK) return st;
+  const DeviceInfo* dev = nullptr;
+  st = device_info(&dev);
+  if (st != SGDB_OK) return st;
+  ArrivalParams p{d_row, row_tag, t, N, P, d_acc, d_counter, d_theta, d_state0, d_state1, d_info, h};
+  const int V = dt == SGDB_BF16 ? 8 : 4;
+  const long long chunks = (P + V - 1) / V;
+  long long grid = (chunks + 255) / 256;
+  const long long cap = static_cast<long long>(dev->sms) * 8;
+  if (grid > cap) grid = cap;
+  if (row_tag != t || grid < 1) grid = 1;  // a wrongly tagged gradient only updates the bookkeeping
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const unsigned g = static_cast<unsigned>(grid);
+#define SGDB_ARRIVAL_CASE(EPV)                                                      \
+  case EPV:                                                                         \
+    if (dt == SGDB_BF16) accumulate_arrival_kernel<BF16, EPV><<<g, 256, 0, s>>>(p); \
+    else accumulate_arrival_kernel<float, EPV><<<g, 256, 0, s>>>(p);                \
+    break;
+  switch (ep) {
+    SGDB_ARRIVAL_CASE(EP_SGD)
+    SGDB_ARRIVAL_CASE(EP_MOMENTUM)
+    SGDB_ARRIVAL_CASE(EP_RMSPROP)
+    SGDB_ARRIVAL_CASE(EP_ADAM)
+    default: return SGDB_ERR_INVALID_ARG;
+  }
+#undef SGDB_ARRIVAL_CASE
+  return launch_status();
+}
+
+// Workspace layout of sgdb_step_host: arrival[W] f32 | tags[W] i32 | order[N] i32 | info[2] i32 |
+// mask[W] u8, rounded up to 256 bytes, then the gradient rows with a 16-byte-multiple pitch.
+static size_t host_ws_header(int32_t N, int32_t b) {
+  const size_t W = static_cast<size_t>(N) + b;
+  const size_t raw = W * 4 + W * 4 + static_cast<size_t>(N) * 4 + 8 + W;
+  return (raw + 255) & ~static_cast<size_t>(255);
+}
+static int64_t host_ws_pitch(sgdb_dtype_t dt, int64_t P) {
+  const int64_t v = dt == SGDB_BF16 ? 8 : 4;
+  return (P + v - 1) / v * v;
+}
+
+size_t sgdb_step_host_workspace_bytes(sgdb_dtype_t dt, int64_t P, int64_t ld, int32_t N, int32_t b) {
+  if (!dtype_ok(dt) || P < 0 || ld < P || N < 1 || b < 0 || static_cast<int64_t>(N) + b > SGDB_MAX_WORKERS)
+    return 0;
+  return host_ws_header(N, b) +
+         static_cast<size_t>(N + b) * static_cast<size_t>(host_ws_pitch(dt, P)) * dtype_size(dt);
+}
+
+sgdb_status_t sgdb_step_host(const void* h_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, const float* h_arrival,
+                             const int32_t* h_tags, int32_t t, int32_t N, int32_t b, float* d_theta,
+                             float* d_state0, float* d_state1, const sgdb_opt_t* opt, float* h_theta_out,
+                             uint8_t* h_mask, int32_t* h_order, int32_t* h_info, void* d_workspace,
+                             size_t workspace_bytes, void* stream) {
+  sgdb_status_t st = check_selection_args(h_arrival, h_tags, N, b, h_mask, h_order, h_info);
+  if (st != SGDB_OK) return st;
+  if (h_grad == nullptr || d_theta == nullptr || d_workspace == nullptr || !dtype_ok(dt) || P < 0 || ld < P)
+    return SGDB_ERR_INVALID_ARG;
+  if (!is_aligned16(d_workspace) || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
+    return SGDB_ERR_INVALID_ARG;
+  const size_t need = sgdb_step_host_workspace_bytes(dt, P, ld, N, b);
+  if (need == 0 || workspace_bytes < need) return SGDB_ERR_INVALID_ARG;
+  Hyper h;
+  int ep = 0;
+  st = prepare_rule(opt, d_state0, d_state1, &h, &ep);
+  if (st != SGDB_OK) return st;
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t W = static_cast<size_t>(N) + b;
+  unsigned char* ws = static_cast<unsigned char*>(d_workspace);
+  float* d_arrival = reinterpret_cast<float*>(ws);
+  int32_t* d_tags = reinterpret_cast<int32_t*>(ws + W * 4);
+  int32_t* d_order = reinterpret_cast<int32_t*>(ws + W * 8);
+  int32_t* d_info = d_order + N;
+  uint8_t* d_mask = reinterpret_cast<uint8_t*>(d_info + 2);
+  unsigned char* d_rows = ws + host_ws_header(N, b);
+  const size_t esize = dtype_size(dt);
+  const int64_t pitch = host_ws_pitch(dt, P);
+
+  bool ok = cudaMemcpyAsync(d_arrival, h_arrival, W * 4, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+            cudaMemcpyAsync(d_tags, h_tags, W * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  if (!ok) return launch_status();
+  st = launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
+  if (st != SGDB_OK) return st;
+  ok = cudaMemcpyAsync(h_info, d_info, 8, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+       cudaStreamSynchronize(s) == cudaSuccess;
+  if (!ok) return launch_status();
+  if (h_info[1] != SGDB_OK) return static_cast<sgdb_status_t>(h_info[1]);
+  ok = cudaMemcpyAsync(h_order, d_order, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+       cudaMemcpyAsync(h_mask, d_mask, W, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+       cudaStreamSynchronize(s) == cudaSuccess;
+  if (!ok) return launch_status();
+
+  if (P > 0) {
+    // only the kept rows cross to the device, each to the slot of its worker id
+    for (int32_t k = 0; k < N; ++k) {
+      const size_t w = static_cast<size_t>(h_order[k]);
+      if (cudaMemcpyAsync(d_rows + w * static_cast<size_t>(pitch) * esize,
+                          static_cast<const unsigned char*>(h_grad) + w * static_cast<size_t>(ld) * esize,
+                          static_cast<size_t>(P) * esize, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return launch_status();
+    }
+    StreamParams p{};
+    p.table = nullptr;
+    p.flat.theta = d_theta;
+    p.flat.state0 = d_state0;
+    p.flat.state1 = d_state1;
+    p.flat.grad = d_rows;
+    p.flat.ld = pitch;
+    p.flat.len = P;
+    p.S = 1;
+    p.N = N;
+    p.order = d_order;
+    p.info = d_info;
+    p.status_out = d_info + 1;
+    p.h = h;
+    st = launch_stream(dt, ep, p, tiles_of(dt, P), s);
+    if (st != SGDB_OK) return st;
+    if (h_theta_out != nullptr &&
+        cudaMemcpyAsync(h_theta_out, d_theta, static_cast<size_t>(P) * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+      return launch_status();
+    if (cudaMemcpyAsync(h_info, d_info, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess) return launch_status();
+  }
+  if (cudaStreamSynchronize(s) != cudaSuccess) return launch_status();
+  return static_cast<sgdb_status_t>(h_info[1]);
+}
+
+sgdb_status_t sgdb_set_tuning(int32_t stages, int32_t ctas_per_sm) {
+  if (stages > 64 || ctas_per_sm > 8) return SGDB_ERR_INVALID_ARG;
+  g_stages = stages > 0 ? (stages < 2 ? 2 : stages) : kDefaultStages;
+  g_ctas_per_sm = ctas_per_sm > 0 ? ctas_per_sm : kDefaultCtasPerSm;
+  return SGDB_OK;
+}
+
+const char* sgdb_strerror(sgdb_status_t status) {
+  switch (status) {
+    case SGDB_OK: return "ok";
+    case SGDB_ERR_INVALID_ARG: return "invalid argument";
+    case SGDB_ERR_INSUFFICIENT: return "fewer than N gradients carry the current iteration tag";
+    case SGDB_ERR_CUDA: return "CUDA runtime or launch error";
+    case SGDB_ERR_UNSUPPORTED: return "unsupported size or configuration";
+    case SGDB_ERR_TIMEOUT: return "a bounded on-chip wait ran out";
+  }
+  return "unknown status";
+}
+
+int sgdb_version(void) { return kVersion; }
+
+}  // extern "C"

@@ -1,0 +1,477 @@
+// Kernels of libsgdb (sm_100a).
+//
+//   select_first_n_kernel   which N of the N+b gradients the server keeps
+//   stream_rows_kernel      masked mean of the kept rows, fused with the optimizer
+//                           rule (or writing the mean), flat or over a segment table
+//   update_kernel           optimizer rule from a given mean
+//   accumulate_arrival_kernel   one arriving gradient: admit or drop, add, fire at N
+//
+// The path is a reduction bound by HBM bandwidth (about a quarter of a flop per
+// byte), so there are no tensor-core instructions here; what matters is bytes in
+// flight per SM, touch-once cache policy and a fixed summation order.
+#pragma once
+
+#include "sgdb_device.cuh"
+
+namespace sgdb {
+
+// ====================================================================== selection
+//
+// One warp.  Worker j is valid when tag[j] == t and its arrival time is finite.
+// The rank of a valid worker w is the number of valid workers that arrive before it,
+// where "before" compares (arrival time, worker id).  Lanes test 32 workers at a
+// time against w's key and the votes are counted with __ballot_sync / __popc.
+// Workers of rank < N are kept; order[rank] = w puts them in arrival sequence.
+__global__ void __launch_bounds__(32) select_first_n_kernel(const float* __restrict__ arrival,
+                                                            const int32_t* __restrict__ tags,
+                                                            int32_t t, int32_t N, int32_t W,
+                                                            uint8_t* __restrict__ mask,
+                                                            int32_t* __restrict__ order,
+                                                            int32_t* __restrict__ info) {
+  __shared__ float s_arrival[SGDB_MAX_WORKERS];
+  __shared__ uint8_t s_valid[SGDB_MAX_WORKERS];
+  const unsigned kAll = 0xffffffffu;
+  const int lane = threadIdx.x;
+  const int slots = (W + 31) / 32;
+
+  int n_valid = 0;
+  for (int k = 0; k < slots; ++k) {
+    const int j = k * 32 + lane;
+    float a = 0.0f;
+    bool valid = false;
+    if (j < W) {
+      a = arrival[j];
+      valid = (tags[j] == t) && isfinite(a);
+      s_arrival[j] = a;
+      s_valid[j] = valid ? 1 : 0;
+    }
+    n_valid += __popc(__ballot_sync(kAll, valid));
+  }
+  __syncwarp();
+  const bool enough = n_valid >= N;
+  if (lane == 0) {
+    info[0] = n_valid;
+    info[1] = enough ? SGDB_OK : SGDB_ERR_INSUFFICIENT;
+  }
+  if (!enough) return;  // mask and order stay as they were
+
+  for (int w = 0; w < W; ++w) {
+    if (!s_valid[w]) {
+      if (lane == 0) mask[w] = 0;
+      continue;
+    }
+    const float aw = s_arrival[w];
+    int rank = 0;
+    for (int k = 0; k < slots; ++k) {
+      const int j = k * 32 + lane;
+      bool before = false;
+      if (j < W && s_valid[j]) {
+        const float aj = s_arrival[j];
+        before = (aj < aw) || (aj == aw && j < w);
+      }
+      rank += __popc(__ballot_sync(kAll, before));
+    }
+    if (lane == 0) {
+      const bool kept = rank < N;
+      mask[w] = kept ? 1 : 0;
+      if (kept) order[rank] = w;
+    }
+  }
+}
+
+// ====================================================================== row streaming
+//
+// Persistent blocks walk over column tiles of TILE = NT*CH*V columns.  For a tile,
+// the N kept rows are added in order[] sequence into fp32 registers; then the tile's
+// slice of theta and optimizer state is updated (or the mean is stored).
+//
+// Row slices reach shared memory through a ring of `stages` buffers filled by 1-D
+// bulk async copies issued by one producer thread; each buffer has a "full"
+// mbarrier (armed with the byte count, completed by the copy engine) and an "empty"
+// mbarrier (one arrival per consumer warp).  The ring keeps running across tiles, so
+// the next tile's rows are already in flight while this tile's epilogue runs.
+//
+// Bulk copies need 16-byte aligned addresses and sizes.  A segment whose gradient
+// base or row pitch is not 16-byte aligned, and the last (< 16 byte) sliver of a
+// ragged tile, are read with ordinary element loads by the consumers instead; the
+// additions happen in the same order either way.
+
+struct StreamParams {
+  const sgdb_segment_t* table;  // device segment table, or nullptr: use `flat`
+  sgdb_segment_t flat;          // with EP_MEAN, flat.theta is where the mean goes
+  int S;                        // entries in `table`
+  int N;                        // rows to add
+  int stages;                   // ring depth
+  const int32_t* order;         // [N] row ids in summation order
+  const int32_t* info;          // optional [2]; info[1] != SGDB_OK: do nothing
+  int32_t* status_out;          // optional: receives SGDB_ERR_TIMEOUT if a wait runs out
+  Hyper h;
+};
+
+template <typename GT>
+struct TileDesc {
+  const GT* grad;  // row 0 of this tile's columns
+  float* theta;    // this tile's slice (mean output for EP_MEAN)
+  float* s0;
+  float* s1;
+  long long ld;
+  int ncols;      // valid columns in the tile
+  int bulk_cols;  // leading columns delivered by bulk copy (0: none)
+  bool vec_ok;    // theta/state slices may be accessed 16 bytes at a time
+};
+
+template <typename GT, int TILE>
+__device__ __forceinline__ TileDesc<GT> locate_tile(const StreamParams& p, const int* prefix_s,
+                                                    int tile) {
+  constexpr int V = GradTraits<GT>::kVec;
+  sgdb_segment_t seg;
+  long long col0;
+  if (p.table == nullptr) {
+    seg = p.flat;
+    col0 = static_cast<long long>(tile) * TILE;
+  } else {
+    int lo = 0, hi = p.S;  // first index whose prefix exceeds `tile`, minus one
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (prefix_s[mid + 1] > tile) hi = mid; else lo = mid + 1;
+    }
+    seg = p.table[lo];
+    col0 = static_cast<long long>(tile - prefix_s[lo]) * TILE;
+  }
+  TileDesc<GT> td;
+  td.grad = static_cast<const GT*>(seg.grad) + col0;
+  td.theta = static_cast<float*>(seg.theta) + col0;
+  td.s0 = seg.state0 ? static_cast<float*>(seg.state0) + col0 : nullptr;
+  td.s1 = seg.state1 ? static_cast<float*>(seg.state1) + col0 : nullptr;
+  td.ld = seg.ld;
+  const long long rest = seg.len - col0;
+  td.ncols = rest < TILE ? static_cast<int>(rest) : TILE;
+  const bool bulk_ok = ((reinterpret_cast<uintptr_t>(seg.grad) & 15u) == 0) &&
+                       (((seg.ld * static_cast<long long>(sizeof(GT))) & 15) == 0);
+  td.bulk_cols = bulk_ok ? (td.ncols / V) * V : 0;
+  td.vec_ok = (((reinterpret_cast<uintptr_t>(seg.theta) | reinterpret_cast<uintptr_t>(seg.state0) |
+                 reinterpret_cast<uintptr_t>(seg.state1)) & 15u) == 0);
+  return td;
+}
+
+template <typename GT, int EP, int NT, int CH>
+__global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamParams p) {
+  using Tr = GradTraits<GT>;
+  using Rule = RuleTraits<EP>;
+  constexpr int V = Tr::kVec;
+  constexpr int TILE = NT * CH * V;
+  constexpr uint32_t STAGE_BYTES = TILE * sizeof(GT);
+  constexpr int NW = NT / 32;
+
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ int s_abort;
+
+  if (p.info != nullptr && p.info[1] != SGDB_OK) return;  // e.g. fewer than N current gradients
+
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const int stages = p.stages;
+  const int N = p.N;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + static_cast<size_t>(stages) * STAGE_BYTES);
+  uint64_t* empty_bar = full_bar + stages;
+  int* order_s = reinterpret_cast<int*>(empty_bar + stages);
+  int* prefix_s = order_s + ((N + 3) & ~3);
+
+  for (int i = tid; i < N; i += NT + 32) order_s[i] = p.order[i];
+  if (tid == 0) {
+    s_abort = 0;
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_addr(full_bar + s), 1);
+      mbar_init(smem_addr(empty_bar + s), NW);
+    }
+    fence_barrier_init();
+  }
+  if (p.table != nullptr) {
+    // tiles per segment, then an inclusive scan: prefix_s[i] = tiles in segments < i
+    for (int i = tid; i < p.S; i += NT + 32) {
+      const long long len = p.table[i].len;
+      prefix_s[i + 1] = len > 0 ? static_cast<int>((len + TILE - 1) / TILE) : 0;
+    }
+    if (tid == 0) prefix_s[0] = 0;
+    __syncthreads();
+    if (tid < 32) {
+      int carry = 0;
+      for (int base = 1; base <= p.S; base += 32) {
+        const int idx = base + lane;
+        int v = idx <= p.S ? prefix_s[idx] : 0;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const int up = __shfl_up_sync(0xffffffffu, v, d);
+          if (lane >= d) v += up;
+        }
+        v += carry;
+        if (idx <= p.S) prefix_s[idx] = v;
+        carry = __shfl_sync(0xffffffffu, v, 31);
+      }
+    }
+  }
+  __syncthreads();
+  const int total_tiles =
+      p.table != nullptr ? prefix_s[p.S] : static_cast<int>((p.flat.len + TILE - 1) / TILE);
+  const uint32_t ring_addr = smem_addr(smem);
+  const uint32_t full_addr = smem_addr(full_bar);
+  const uint32_t empty_addr = smem_addr(empty_bar);
+  bool timed_out = false;
+
+  if (tid >= NT) {
+    // ------------------------------------------------------------ producer (one thread)
+    if (tid == NT) {
+      const uint64_t policy = l2_policy_evict_first();  // rows are read exactly once
+      int s = 0;
+      uint32_t phase = 0;
+      for (int tile = blockIdx.x; tile < total_tiles && !timed_out; tile += gridDim.x) {
+        const TileDesc<GT> td = locate_tile<GT, TILE>(p, prefix_s, tile);
+        if (td.bulk_cols == 0) continue;
+        const uint32_t bytes = static_cast<uint32_t>(td.bulk_cols) * sizeof(GT);
+        for (int k = 0; k < N; ++k) {
+          if (!mbar_wait(empty_addr + 8u * s, phase ^ 1u, &s_abort)) {
+            timed_out = true;
+            break;
+          }
+          const GT* src = td.grad + static_cast<long long>(order_s[k]) * td.ld;
+          mbar_arrive_expect_tx(full_addr + 8u * s, bytes);
+          bulk_copy_g2s(ring_addr + static_cast<uint32_t>(s) * STAGE_BYTES, src, bytes,
+                        full_addr + 8u * s, policy);
+          if (++s == stages) {
+            s = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ consumers
+    const float n_as_float = static_cast<float>(N);
+    int s = 0;
+    uint32_t phase = 0;
+    for (int tile = blockIdx.x; tile < total_tiles && !timed_out; tile += gridDim.x) {
+      const TileDesc<GT> td = locate_tile<GT, TILE>(p, prefix_s, tile);
+
+      // theta and state of this tile are requested now and used after the row loop
+      float th[CH][V], s0[CH][V], s1[CH][V];
+#pragma unroll
+      for (int c = 0; c < CH; ++c) {
+        const int o = (tid + c * NT) * V;
+        const int n = td.ncols - o;
+        if (n > 0) {
+          const bool vec = td.vec_ok && n >= V;
+          if (Rule::kTheta) load_floats<V>(td.theta + o, vec, n, th[c]);
+          if (Rule::kState0) load_floats<V>(td.s0 + o, vec, n, s0[c]);
+          if (Rule::kState1) load_floats<V>(td.s1 + o, vec, n, s1[c]);
+        }
+      }
+
+      float acc[CH][V];
+#pragma unroll
+      for (int c = 0; c < CH; ++c)
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[c][e] = 0.0f;
+
+      for (int k = 0; k < N; ++k) {
+        const GT* row = td.grad + static_cast<long long>(order_s[k]) * td.ld;
+        const unsigned char* stage = smem + static_cast<size_t>(s) * STAGE_BYTES;
+        if (td.bulk_cols > 0) {
+          if (!mbar_wait(full_addr + 8u * s, phase, &s_abort)) {
+            timed_out = true;
+            break;
+          }
+        }
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+          const int o = (tid + c * NT) * V;
+          if (o + V <= td.bulk_cols) {
+            const uint4 v = *reinterpret_cast<const uint4*>(stage + static_cast<size_t>(o) * sizeof(GT));
+            float x[V];
+            Tr::unpack(v, x);
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[c][e] = __fadd_rn(acc[c][e], x[e]);
+          } else if (o < td.ncols) {
+#pragma unroll
+            for (int e = 0; e < V; ++e)
+              if (o + e < td.ncols) acc[c][e] = __fadd_rn(acc[c][e], Tr::widen(row[o + e]));
+          }
+        }
+        if (td.bulk_cols > 0) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty_addr + 8u * s);
+          if (++s == stages) {
+            s = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+      if (timed_out) break;
+
+#pragma unroll
+      for (int c = 0; c < CH; ++c) {
+        const int o = (tid + c * NT) * V;
+        const int n = td.ncols - o;
+        if (n > 0) {
+          const bool vec = td.vec_ok && n >= V;
+          float g[V];
+#pragma unroll
+          for (int e = 0; e < V; ++e) g[e] = __fdiv_rn(acc[c][e], n_as_float);
+          if (EP == EP_MEAN) {
+            store_floats<V>(td.theta + o, vec, n, g);
+          } else {
+#pragma unroll
+            for (int e = 0; e < V; ++e) apply_rule<EP>(p.h, g[e], th[c][e], s0[c][e], s1[c][e]);
+            store_floats<V>(td.theta + o, vec, n, th[c]);
+            if (Rule::kState0) store_floats<V>(td.s0 + o, vec, n, s0[c]);
+            if (Rule::kState1) store_floats<V>(td.s1 + o, vec, n, s1[c]);
+          }
+        }
+      }
+    }
+  }
+  if (timed_out && p.status_out != nullptr) *p.status_out = SGDB_ERR_TIMEOUT;
+}
+
+// ====================================================================== update from a mean
+
+struct UpdateParams {
+  float* theta;
+  float* s0;
+  float* s1;
+  const float* mean;
+  long long P;
+  const int32_t* info;
+  Hyper h;
+};
+
+template <int EP>
+__global__ void __launch_bounds__(256) update_kernel(const UpdateParams p) {
+  using Rule = RuleTraits<EP>;
+  if (p.info != nullptr && p.info[1] != SGDB_OK) return;
+  const long long chunks = (p.P + 3) / 4;
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  for (long long q = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; q < chunks; q += stride) {
+    const long long i = q * 4;
+    const long long rest = p.P - i;
+    const int n = rest < 4 ? static_cast<int>(rest) : 4;
+    const bool vec = n == 4;
+    float g[4], th[4], s0[4], s1[4];
+    load_floats<4>(p.mean + i, vec, n, g);
+    load_floats<4>(p.theta + i, vec, n, th);
+    if (Rule::kState0) load_floats<4>(p.s0 + i, vec, n, s0);
+    if (Rule::kState1) load_floats<4>(p.s1 + i, vec, n, s1);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) apply_rule<EP>(p.h, g[e], th[e], s0[e], s1[e]);
+    store_floats<4>(p.theta + i, vec, n, th);
+    if (Rule::kState0) store_floats<4>(p.s0 + i, vec, n, s0);
+    if (Rule::kState1) store_floats<4>(p.s1 + i, vec, n, s1);
+  }
+}
+
+// ====================================================================== one arrival
+//
+// Every block reads the server state {accepted, seen, ticket, lowest open iteration}
+// before doing anything and takes the same decision from it.  The state is only
+// changed by the block that finishes last (it holds the last ticket), i.e. after
+// every block has read it, so one launch needs neither a grid-wide barrier nor a
+// wait.  The next arrival's launch is ordered after this one by the stream.
+
+struct ArrivalParams {
+  const void* row;
+  int32_t row_tag, t, N;
+  long long P;
+  float* acc;
+  int32_t* counter;  // [4]
+  float* theta;
+  float* s0;
+  float* s1;
+  int32_t* info;  // [2]
+  Hyper h;
+};
+
+template <typename GT, int EP>
+__global__ void __launch_bounds__(256) accumulate_arrival_kernel(const ArrivalParams p) {
+  using Tr = GradTraits<GT>;
+  using Rule = RuleTraits<EP>;
+  constexpr int V = Tr::kVec;
+  __shared__ int s_accepted, s_open;
+  if (threadIdx.x == 0) {
+    s_accepted = *reinterpret_cast<volatile int32_t*>(p.counter + 0);
+    s_open = *reinterpret_cast<volatile int32_t*>(p.counter + 3);
+  }
+  __syncthreads();
+  const int accepted = s_accepted;
+  const bool admit = (p.row_tag == p.t) && (p.t >= s_open) && (accepted < p.N);
+  const bool first = accepted == 0;          // the set was empty: start the sum from +0
+  const bool last = accepted + 1 == p.N;     // this gradient completes the set
+
+  if (admit) {
+    const GT* row = static_cast<const GT*>(p.row);
+    const bool row_vec = (reinterpret_cast<uintptr_t>(p.row) & 15u) == 0;
+    const float n_as_float = static_cast<float>(p.N);
+    const long long chunks = (p.P + V - 1) / V;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long q = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; q < chunks; q += stride) {
+      const long long i = q * V;
+      const long long rest = p.P - i;
+      const int n = rest < V ? static_cast<int>(rest) : V;
+      const bool vec = n == V;
+      float x[V], a[V];
+      if (vec && row_vec) {
+        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(row + i));
+        Tr::unpack(v, x);
+      } else {
+#pragma unroll
+        for (int e = 0; e < V; ++e) x[e] = e < n ? Tr::widen(row[i + e]) : 0.0f;
+      }
+      if (first) {
+#pragma unroll
+        for (int e = 0; e < V; ++e) a[e] = 0.0f;
+      } else {
+        load_floats<V>(p.acc + i, vec, n, a);
+      }
+#pragma unroll
+      for (int e = 0; e < V; ++e) a[e] = __fadd_rn(a[e], x[e]);
+      if (!last) {
+        store_floats<V>(p.acc + i, vec, n, a);
+      } else {
+        float th[V], s0[V], s1[V];
+        load_floats<V>(p.theta + i, vec, n, th);
+        if (Rule::kState0) load_floats<V>(p.s0 + i, vec, n, s0);
+        if (Rule::kState1) load_floats<V>(p.s1 + i, vec, n, s1);
+#pragma unroll
+        for (int e = 0; e < V; ++e)
+          apply_rule<EP>(p.h, __fdiv_rn(a[e], n_as_float), th[e], s0[e], s1[e]);
+        store_floats<V>(p.theta + i, vec, n, th);
+        if (Rule::kState0) store_floats<V>(p.s0 + i, vec, n, s0);
+        if (Rule::kState1) store_floats<V>(p.s1 + i, vec, n, s1);
+      }
+    }
+  }
+
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned ticket = atomicAdd(reinterpret_cast<unsigned*>(p.counter + 2), 1u);
+    if (ticket == gridDim.x - 1) {  // every block has read the state: now it may change
+      p.counter[2] = 0;
+      p.counter[1] += 1;
+      int outcome = 0, after = accepted;
+      if (admit) {
+        after = accepted + 1;
+        outcome = 1;
+        if (last) {
+          outcome = 2;
+          p.counter[0] = 0;
+          p.counter[3] = p.t + 1;
+        } else {
+          p.counter[0] = after;
+        }
+      }
+      p.info[0] = outcome;
+      p.info[1] = after;
+    }
+  }
+}
+
+}  // namespace sgdb

@@ -1,0 +1,92 @@
+"""The C-ABI library builds, loads and exports every symbol include/sgdb.h declares (no GPU needed)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_1604_00981_b200 import build
+
+    return ctypes.CDLL(build.build())
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "sgdb.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sgdb_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared()
+    assert {"sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented",
+            "sgdb_accumulate_arrival", "sgdb_step_host"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_binding_exposes_the_same_names():
+    from paper_1604_00981_b200 import binding
+
+    for n in _declared():
+        assert callable(getattr(binding, n)), n
+    assert set(binding.EXPORTS) == set(_declared())
+
+
+def test_version_and_strerror(lib):
+    lib.sgdb_strerror.restype = ctypes.c_char_p
+    assert lib.sgdb_version() >= 100
+    seen = {lib.sgdb_strerror(i) for i in range(6)}
+    assert len(seen) == 6 and all(seen)
+    assert lib.sgdb_strerror(99)
+
+
+def test_host_checkable_errors_return_before_any_launch(lib):
+    """Null pointers and impossible sizes are refused on the host (no CUDA call is made)."""
+    null = ctypes.c_void_p(0)
+    one = ctypes.c_void_p(16)  # a non-null, 16-byte aligned stand-in that is never dereferenced
+    i32, i64 = ctypes.c_int32, ctypes.c_int64
+    INVALID = 1
+    assert lib.sgdb_select(null, one, i32(0), i32(1), i32(0), one, one, one, null) == INVALID
+    assert lib.sgdb_select(one, one, i32(0), i32(0), i32(0), one, one, one, null) == INVALID  # N < 1
+    assert lib.sgdb_select(one, one, i32(0), i32(1), i32(-1), one, one, one, null) == INVALID  # b < 0
+    assert lib.sgdb_select(one, one, i32(0), i32(1000), i32(25), one, one, one, null) == INVALID  # W > 1024
+    assert lib.sgdb_aggregate(one, i32(0), i64(10), i64(9), i32(1), one, null, one, null) == INVALID  # ld < P
+    assert lib.sgdb_aggregate(ctypes.c_void_p(20), i32(0), i64(10), i64(10), i32(1), one, null, one, null) == INVALID
+    assert lib.sgdb_aggregate(one, i32(7), i64(10), i64(10), i32(1), one, null, one, null) == INVALID  # dtype
+    assert lib.sgdb_update(one, null, null, one, i64(4), null, null, null) == INVALID  # no optimizer
+    lib.sgdb_step_host_workspace_bytes.restype = ctypes.c_size_t
+    assert lib.sgdb_step_host_workspace_bytes(i32(0), i64(-1), i64(0), i32(1), i32(0)) == 0
+    need = lib.sgdb_step_host_workspace_bytes(i32(0), i64(10), i64(10), i32(5), i32(1))
+    assert need >= 6 * 12 * 4
+    assert lib.sgdb_set_tuning(i32(1000), i32(0)) == INVALID
+    assert lib.sgdb_set_tuning(i32(0), i32(0)) == 0
+
+
+def test_optimizer_argument_checks(lib):
+    from paper_1604_00981_b200.binding import _COpt
+
+    one = ctypes.c_void_p(16)
+    null = ctypes.c_void_p(0)
+    i64 = ctypes.c_int64
+    bad_kind = _COpt(9, 0.1, 0, 0, 0, 0, 0, 1)
+    assert lib.sgdb_update(one, null, null, one, i64(4), ctypes.byref(bad_kind), null, null) == 1
+    momentum_without_state = _COpt(1, 0.1, 0.9, 0, 0, 0, 0, 1)
+    assert lib.sgdb_update(one, null, null, one, i64(4), ctypes.byref(momentum_without_state), null, null) == 1
+    adam_step0 = _COpt(3, 0.1, 0, 0, 0.9, 0.999, 1e-8, 0)
+    assert lib.sgdb_update(one, one, one, one, i64(4), ctypes.byref(adam_step0), null, null) == 1
+    nan_lr = _COpt(0, float("nan"), 0, 0, 0, 0, 0, 1)
+    assert lib.sgdb_update(one, null, null, one, i64(4), ctypes.byref(nan_lr), null, null) == 1
+
+
+def test_graft_entry_build():
+    import __graft_entry__
+
+    __graft_entry__.build()
+    from paper_1604_00981_b200 import build
+
+    assert os.path.exists(build.LIB) and not build.is_stale()

@@ -1,0 +1,252 @@
+"""Parity of the multi-tensor step, the arrival-by-arrival mode and the host-buffer step with the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import (OPTS, TOL_BF16, TOL_F32, gpu_opt, gpu_state, oracle_opt, oracle_state, rel_err,
+                     selection_buffers, step_inputs, to_dev)
+from paper_1604_00981_b200 import workload as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sgdb(cuda_device):
+    from paper_1604_00981_b200 import binding
+
+    return binding
+
+
+# ------------------------------------------------------------------ multi-tensor (segment table)
+
+
+def _make_model(dev, lengths, W, kind, dtype, seed, packed):
+    """Tensors of the given lengths.  packed=False: every tensor has its own allocation and a row pitch
+    padded to 16 bytes.  packed=True: parameters, state and gradients of all tensors are carved out of
+    shared buffers back to back, so most tensors start at an address that is only element-aligned."""
+    scales = wl.worker_scales(seed, W)
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    vec = 4 if dtype == "f32" else 8
+    segs = []
+    total = int(sum(lengths))
+    if packed:
+        th_all = wl.theta0(seed, total, dev)
+        s_all = [torch.zeros(total, device=dev) for _ in range(2)]
+        g_all = torch.empty(W * total, dtype=tdt, device=dev)
+    off = 0
+    for i, L in enumerate(int(x) for x in lengths):
+        if packed:
+            theta = th_all[off:off + L]
+            s0, s1 = s_all[0][off:off + L], s_all[1][off:off + L]
+            grad = g_all[W * off:W * (off + L)].view(W, L)
+            wl.grad_matrix(seed + i, 0, W, L, scales, dtype, dev, out=grad)
+        else:
+            theta = wl.theta0(seed + i, L, dev)
+            s0, s1 = torch.zeros(L, device=dev), torch.zeros(L, device=dev)
+            ld = (L + vec - 1) // vec * vec
+            grad = wl.grad_matrix(seed + i, 0, W, L, scales, dtype, dev, ld=ld, pad_value=float("nan"))
+        n = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2}[kind]
+        segs.append((theta, s0 if n >= 1 else None, s1 if n >= 2 else None, grad))
+        off += L
+    return segs, scales
+
+
+def _regen(segs, scales, seed, t, W, dtype, dev, packed):
+    for i, (theta, _, _, grad) in enumerate(segs):
+        L = theta.numel()
+        if packed:
+            wl.grad_matrix(seed + i, t, W, L, scales, dtype, dev, out=grad)
+        else:
+            wl.grad_matrix(seed + i, t, W, L, scales, dtype, dev, ld=grad.stride(0), out=grad, pad_value=float("nan"))
+
+
+@pytest.mark.parametrize("packed", [False, True])
+@pytest.mark.parametrize("kind,dtype", [("momentum", "f32"), ("adam", "bf16"), ("sgd", "f32"), ("rmsprop", "bf16")])
+def test_segmented_step_matches_oracle_and_per_tensor_launches(sgdb, cuda_device, kind, dtype, packed):
+    dev = cuda_device
+    W, N, T, seed = 14, 11, 3, 101
+    rng = np.random.default_rng(seed)
+    # log-uniform lengths like the 300-tensor workload, scaled down; plus the awkward ones
+    lengths = np.floor(np.exp(rng.uniform(np.log(1), np.log(30_000), size=60))).astype(np.int64).tolist()
+    lengths += [1, 2, 3, 4, 5, 7, 8, 2047, 2048, 2049, 4096, 4097, 0, 6145]
+    segs, scales = _make_model(dev, lengths, W, kind, dtype, seed, packed)
+    twins = [tuple(None if x is None else x.clone() for x in s[:3]) for s in segs]  # per-tensor launches
+    th_o = [s[0].cpu().numpy().astype(np.float64) for s in segs]
+    st_o = [oracle_state(kind, len(x)) for x in th_o]
+    table = sgdb.make_segment_table(segs, dev)
+    mask, order, info = selection_buffers(W, N, dev)
+    mask2, order2, info2 = selection_buffers(W, N, dev)
+    tol = TOL_F32 if dtype == "f32" else TOL_BF16
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    for t in range(T):
+        if t:
+            _regen(segs, scales, seed, t, W, dtype, dev, packed)
+        arrival, tags = step_inputs(seed, t, W, N)
+        a_d, t_d = to_dev(arrival, dev), to_dev(tags, dev)
+        sgdb.sgdb_step_segmented(table, len(segs), tdt, a_d, t_d, t, N, W - N, gpu_opt(OPTS[kind], t + 1),
+                                 mask, order, info)
+        rc, mask_o, order_o, n_valid = oracle.select(arrival, tags, t, N, W - N)
+        assert rc == oracle.OK and info.cpu().tolist() == [n_valid, 0]
+        assert order.cpu().numpy().tolist() == order_o.tolist() and mask.cpu().numpy().tolist() == mask_o.tolist()
+        for i, (theta, s0, s1, grad) in enumerate(segs):
+            L = theta.numel()
+            if L == 0:
+                continue
+            aligned = all(x is None or x.data_ptr() % 16 == 0 for x in (theta, s0, s1, grad))
+            if aligned:  # the flat call wants 16-byte aligned bases; compare bit for bit where it applies
+                sgdb.sgdb_step(grad, L, a_d, t_d, t, N, W - N, twins[i][0], twins[i][1], twins[i][2],
+                               gpu_opt(OPTS[kind], t + 1), mask2, order2, info2, ld=grad.stride(0))
+                assert torch.equal(theta, twins[i][0]), (i, L)
+            mean = oracle.aggregate(wl.as_oracle_array(grad), L, order_o, ld=grad.stride(0))
+            oracle.update(th_o[i], st_o[i][0], st_o[i][1], mean, oracle_opt(OPTS[kind], t + 1))
+    for i, (theta, s0, s1, _) in enumerate(segs):
+        if theta.numel() == 0:
+            continue
+        # tiny tensors: compare against the model-wide scale, not the tensor's own rms
+        scale = max(1.0, float(np.sqrt(np.mean(th_o[i] ** 2))))
+        assert np.max(np.abs(theta.cpu().numpy() - th_o[i])) / scale < tol * 4, (i, theta.numel())
+        if theta.numel() >= 64:
+            assert rel_err(theta.cpu().numpy(), th_o[i]) < tol, (i, theta.numel())
+            if s0 is not None:
+                assert rel_err(s0.cpu().numpy(), st_o[i][0]) < tol
+            if s1 is not None:
+                assert rel_err(s1.cpu().numpy(), st_o[i][1]) < tol
+
+
+def test_segmented_edge_cases(sgdb, cuda_device):
+    dev = cuda_device
+    W, N = 4, 3
+    mask, order, info = selection_buffers(W, N, dev)
+    a_d = to_dev(np.array([1, 2, 3, 4], np.float32), dev)
+    t_d = torch.zeros(W, dtype=torch.int32, device=dev)
+    # an empty table is a selection only
+    empty = torch.empty(0, dtype=torch.uint8, device=dev)
+    keep = torch.zeros(48, dtype=torch.uint8, device=dev)
+    sgdb.sgdb_step_segmented(keep, 0, torch.float32, a_d, t_d, 0, N, 1, gpu_opt(OPTS["sgd"]), mask, order, info)
+    assert info.cpu().tolist() == [4, 0] and order.cpu().tolist() == [0, 1, 2]
+    del empty
+    with pytest.raises(sgdb.SgdbError) as e:
+        sgdb.sgdb_step_segmented(keep, sgdb.SGDB_MAX_SEGMENTS + 1, torch.float32, a_d, t_d, 0, N, 1,
+                                 gpu_opt(OPTS["sgd"]), mask, order, info)
+    assert e.value.status == sgdb.SGDB_ERR_UNSUPPORTED
+    # the largest table, every tensor tiny
+    S = sgdb.SGDB_MAX_SEGMENTS
+    theta = torch.zeros(S * 3, device=dev)
+    grad = torch.ones((S, W, 3), device=dev)
+    segs = [(theta[3 * i:3 * i + 3], None, None, grad[i]) for i in range(S)]
+    table = sgdb.make_segment_table(segs, dev)
+    sgdb.sgdb_step_segmented(table, S, torch.float32, a_d, t_d, 0, N, 1, gpu_opt(dict(kind="sgd", lr=0.5)),
+                             mask, order, info)
+    assert info.cpu().tolist() == [4, 0]
+    assert (theta == -0.5).all()
+
+
+# ------------------------------------------------------------------ arrival by arrival
+
+
+@pytest.mark.parametrize("kind,dtype,P,b", [("rmsprop", "f32", 100_003, 0), ("rmsprop", "f32", 100_003, 2),
+                                            ("rmsprop", "f32", 65_536, 4), ("rmsprop", "f32", 100_003, 8),
+                                            ("adam", "bf16", 50_001, 3), ("sgd", "f32", 5, 1),
+                                            ("momentum", "bf16", 4099, 2)])
+def test_accumulate_on_arrival(sgdb, cuda_device, kind, dtype, P, b):
+    """Rows are delivered one per call in arrival sequence, stale rows and late rows included.  Outcomes
+    and counts match the oracle's replay of Algorithm 4; parameters match the oracle within tolerance
+    and the fused step bit for bit."""
+    dev = cuda_device
+    N, T, seed = 12, 3, 111 + b
+    W = N + b
+    scales = wl.worker_scales(seed, W)
+    theta = wl.theta0(seed, P, dev)
+    theta_f = theta.clone()
+    s0, s1 = gpu_state(kind, P, dev)
+    sf = gpu_state(kind, P, dev)
+    acc = torch.full((P,), float("nan"), device=dev)  # needs no clearing by the caller
+    counter = torch.zeros(4, dtype=torch.int32, device=dev)
+    info = torch.zeros(2, dtype=torch.int32, device=dev)
+    th_o = theta.cpu().numpy().astype(np.float64)
+    s0_o, s1_o = oracle_state(kind, P)
+    acc_o, state_o = np.zeros(P), oracle.new_server_state()
+    mask, order, finfo = selection_buffers(W, N, dev)
+    seen = 0
+    late = None
+    for t in range(T):
+        grad = wl.grad_matrix(seed, t, W, P, scales, dtype, dev)
+        grad_h = wl.as_oracle_array(grad)
+        arrival, tags = step_inputs(seed, t, W, N + 0)
+        stale = int(np.argsort(arrival, kind="stable")[1])
+        if b >= 2 and int((tags == t).sum()) - int(tags[stale] == t) >= N:
+            tags[stale] = t - 1  # an early arrival that is stale
+        opt, opt_o = gpu_opt(OPTS[kind], t + 1), oracle_opt(OPTS[kind], t + 1)
+        deliveries = [(grad[w], grad_h[w], int(tags[w])) for w in wl.delivery_sequence(arrival)]
+        if late is not None:
+            deliveries.insert(1, late)  # a straggler of the previous iteration turns up now
+        outcomes = []
+        for row, row_h, tag in deliveries:
+            sgdb.sgdb_accumulate_arrival(row, tag, t, N, acc, counter, theta, s0, s1, opt, info)
+            want = oracle.accumulate_arrival(row_h, tag, t, N, acc_o, state_o, th_o, s0_o, s1_o, opt_o)
+            seen += 1
+            got = info.cpu().tolist()
+            assert got[0] == want
+            c = counter.cpu().tolist()
+            assert c[0] == state_o[0] and c[1] == seen == state_o[1] and c[2] == 0 and c[3] == state_o[2]
+            assert got[1] == (N if want == 2 else state_o[0])
+            outcomes.append(want)
+        assert outcomes.count(2) == 1 and outcomes.count(1) == N - 1
+        assert all(o == 0 for o in outcomes[outcomes.index(2) + 1:])  # the slowest are dropped when they arrive
+        sgdb.sgdb_step(grad, P, to_dev(arrival, dev), to_dev(tags, dev), t, N, b, theta_f, sf[0], sf[1], opt,
+                       mask, order, finfo)
+        assert torch.equal(theta, theta_f)
+        late = (grad[int(order[-1])].clone(), grad_h[int(order[-1])].copy(), t)
+    tol = TOL_F32 if dtype == "f32" else TOL_BF16
+    assert rel_err(theta.cpu().numpy(), th_o) < tol
+    for x, y in ((s0, s0_o), (s1, s1_o)):
+        assert x is None or rel_err(x.cpu().numpy(), y) < tol
+    for x, y in zip((s0, s1), sf):
+        assert x is None or torch.equal(x, y)
+
+
+# ------------------------------------------------------------------ gradients in host memory
+
+
+@pytest.mark.parametrize("dtype,P,pad,pinned", [("f32", 70_001, 0, True), ("bf16", 70_001, 5, False), ("f32", 3, 0, False)])
+def test_step_with_host_gradients(sgdb, cuda_device, dtype, P, pad, pinned):
+    dev = cuda_device
+    W, N, T, seed, kind = 18, 15, 3, 121, "rmsprop"
+    ld = P + pad
+    scales = wl.worker_scales(seed, W)
+    theta = wl.theta0(seed, P, dev)
+    theta_d = theta.clone()
+    s0, s1 = gpu_state(kind, P, dev)
+    sd = gpu_state(kind, P, dev)
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    ws = torch.empty(sgdb.sgdb_step_host_workspace_bytes(tdt, P, ld, N, W - N), dtype=torch.uint8, device=dev)
+    h_theta = torch.empty(P, dtype=torch.float32)
+    h_mask = torch.empty(W, dtype=torch.uint8)
+    h_order = torch.empty(N, dtype=torch.int32)
+    h_info = torch.empty(2, dtype=torch.int32)
+    mask, order, info = selection_buffers(W, N, dev)
+    for t in range(T):
+        grad = wl.grad_matrix(seed, t, W, P, scales, dtype, dev, ld=ld)
+        h_grad = grad.cpu()
+        if pinned:
+            h_grad = h_grad.pin_memory()
+        arrival, tags = step_inputs(seed, t, W, N)
+        st = sgdb.sgdb_step_host(h_grad, P, torch.from_numpy(arrival), torch.from_numpy(tags), t, N, W - N,
+                                 theta, s0, s1, gpu_opt(OPTS[kind], t + 1), h_theta, h_mask, h_order, h_info, ws,
+                                 ld=ld)
+        assert st == 0
+        sgdb.sgdb_step(grad, P, to_dev(arrival, dev), to_dev(tags, dev), t, N, W - N, theta_d, sd[0], sd[1],
+                       gpu_opt(OPTS[kind], t + 1), mask, order, info, ld=ld)
+        assert torch.equal(theta, theta_d) and torch.equal(h_theta, theta.cpu())
+        assert torch.equal(h_order, order.cpu()) and torch.equal(h_mask, mask.cpu())
+        assert h_info.tolist() == info.cpu().tolist()
+    # too few current gradients: reported as the return value, nothing changes
+    tags = np.full(W, 99, np.int32)
+    before = theta.clone()
+    st = sgdb.sgdb_step_host(h_grad, P, torch.from_numpy(arrival), torch.from_numpy(tags), 5, N, W - N, theta, s0, s1,
+                             gpu_opt(OPTS[kind]), h_theta, h_mask, h_order, h_info, ws, ld=ld)
+    assert st == sgdb.SGDB_ERR_INSUFFICIENT and torch.equal(theta, before)
+    with pytest.raises(sgdb.SgdbError):  # workspace too small
+        sgdb.sgdb_step_host(h_grad, P, torch.from_numpy(arrival), torch.from_numpy(tags), 5, N, W - N, theta, s0, s1,
+                            gpu_opt(OPTS[kind]), h_theta, h_mask, h_order, h_info, ws[:256], ld=ld)
