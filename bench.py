@@ -228,6 +228,8 @@ def run_native(args, cfg):
     assert bool(torch.isfinite(theta).all())
 
     # ---- end to end: gradients start in pinned host memory, new parameters are read back
+    if args.no_e2e:
+        return finish(args, cfg, dist, dev, rank, world, ms_total, None, 0, clocks, grad_bytes, total_bytes, esize)
     e2e_steps = max(1, min(args.steps, 3))
     ws = torch.empty(sgdb.sgdb_step_host_workspace_bytes(grad.dtype, P, P, N, b), dtype=torch.uint8, device=dev)
     h_grad = torch.empty((W, P), dtype=grad.dtype, pin_memory=True)
@@ -255,16 +257,24 @@ def run_native(args, cfg):
     e_stop.record()
     barrier()
     e2e_ms = e_start.elapsed_time(e_stop)
+    return finish(args, cfg, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks, grad_bytes, total_bytes, esize)
 
+
+def finish(args, cfg, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks, grad_bytes, total_bytes, esize):
+    W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
     # ---- max over ranks
     if dist is not None:
-        tt = torch.tensor([ms_total, e2e_ms], device=dev, dtype=torch.float64)
+        tt = torch.tensor([ms_total, e2e_ms or 0.0], device=dev, dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total, e2e_ms = float(tt[0]), float(tt[1])
+        ms_total, e2e_ms = float(tt[0]), (float(tt[1]) if e2e_ms is not None else None)
     ms_per_step = ms_total / args.steps
     value = world * grad_bytes / (ms_per_step * 1e-3) / 1e9
     total_gbs_per_gpu = total_bytes / (ms_per_step * 1e-3) / 1e9
-    e2e_value = world * grad_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9
+    e2e = None
+    if e2e_ms is not None:
+        e2e = {"value": world * grad_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": N * P * esize + W * 8, "d2h_bytes_per_step": P * 4 + W + N * 4 + 16,
+               "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps}
 
     if rank == 0:
         peak, peak_kind = measured_hbm_peak()
@@ -294,9 +304,7 @@ def run_native(args, cfg):
                          "frac": total_gbs_per_gpu / peak, "traffic": traffic, "peak_source": peak_kind,
                          "kernel": "stream_rows_kernel<float, rmsprop> (duration = whole step, including the one-warp select launch)",
                          "algorithmic_bytes_per_launch": total_bytes},
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": N * P * esize + W * 8,
-                    "d2h_bytes_per_step": P * 4 + W + N * 4 + 16, "steps": e2e_steps,
-                    "ms_per_step": e2e_ms / e2e_steps},
+            "e2e": e2e,
             "gpu_launches": 2 * args.steps,
             "clocks": clocks.summary(),
             "cpu_baseline": cpu,
@@ -313,10 +321,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["native", "reference"], default="native")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--columns", type=int, default=0,
+                    help="override P with a smaller column count (profiler captures); not the benchmark workload")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "native":
         args.warmup = 3
     cfg = wl.CONFIGS[1]
+    if args.columns > 0:
+        import dataclasses
+
+        cfg = dataclasses.replace(cfg, P=args.columns, name=cfg.name + "_columns_%d" % args.columns)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

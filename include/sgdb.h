@@ -177,7 +177,8 @@ sgdb_status_t sgdb_step_segmented(const sgdb_segment_t *d_segments, int32_t S, s
  * sgdb_accumulate_arrival -- Algorithm 4's inner loop taken literally: one
  * gradient per call, in the order the gradients reach the server.
  *
- *   d_row     [P] of type dt   the arriving gradient
+ *   d_row     [P] of type dt   the arriving gradient; any element-aligned address (a row of
+ *                              a matrix with an odd pitch is fine), 16-byte aligned is faster
  *   row_tag, t                 its tag and the server's iteration
  *   d_acc     [P] fp32         running sum, owned by the caller; needs no clearing:
  *                              the first accepted arrival of an iteration overwrites it

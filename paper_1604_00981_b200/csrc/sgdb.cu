@@ -22,7 +22,7 @@ constexpr int kMaxDevices = 64;
 constexpr int kNT = 256;
 constexpr int kCH = 2;
 constexpr int kStageBytes = kNT * kCH * 16;
-constexpr int kDefaultStages = 12;
+constexpr int kDefaultStages = 6;
 constexpr int kDefaultCtasPerSm = 2;
 
 struct DeviceInfo {
@@ -177,7 +177,14 @@ long long tiles_of(int dt, long long len) {
 
 sgdb_status_t launch_select(const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t N, int32_t b,
                             uint8_t* d_mask, int32_t* d_order, int32_t* d_info, cudaStream_t stream) {
-  select_first_n_kernel<<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, N + b, d_mask, d_order, d_info);
+  const int W = N + b;
+  // the kernel is instantiated for 1, 2, 4, ... workers per lane; take the smallest that holds W
+  if (W <= 32) select_first_n_kernel<1><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
+  else if (W <= 64) select_first_n_kernel<2><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
+  else if (W <= 128) select_first_n_kernel<4><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
+  else if (W <= 256) select_first_n_kernel<8><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
+  else if (W <= 512) select_first_n_kernel<16><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
+  else select_first_n_kernel<32><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
   return launch_status();
 }
 
@@ -321,8 +328,7 @@ sgdb_status_t sgdb_accumulate_arrival(const void* d_row, sgdb_dtype_t dt, int32_
   if (d_row == nullptr || d_acc == nullptr || d_counter == nullptr || d_theta == nullptr || d_info == nullptr)
     return SGDB_ERR_INVALID_ARG;
   if (!dtype_ok(dt) || N < 1 || P < 0) return SGDB_ERR_INVALID_ARG;
-  if (!is_aligned16(d_acc) || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1) ||
-      !is_aligned16(d_row))
+  if (!is_aligned16(d_acc) || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
     return SGDB_ERR_INVALID_ARG;
   Hyper h;
   int ep = 0;

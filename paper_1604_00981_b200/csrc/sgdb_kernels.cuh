@@ -19,35 +19,41 @@ namespace sgdb {
 //
 // One warp.  Worker j is valid when tag[j] == t and its arrival time is finite.
 // The rank of a valid worker w is the number of valid workers that arrive before it,
-// where "before" compares (arrival time, worker id).  Lanes test 32 workers at a
-// time against w's key and the votes are counted with __ballot_sync / __popc.
-// Workers of rank < N are kept; order[rank] = w puts them in arrival sequence.
+// where "before" compares (arrival time, worker id).  Workers of rank < N are kept;
+// order[rank] = w puts them in arrival sequence.
+//
+// Lane l keeps workers l, l + 32, ... (SLOTS of them) in registers.  Candidates are
+// taken one at a time: the owning lane broadcasts its key with __shfl_sync, every
+// lane tests its own workers against it, and the votes are counted with
+// __ballot_sync / __popc.  All loops over slots are unrolled, so the single warp has
+// enough independent work in flight to hide its own latencies.  Each lane remembers
+// the ranks of its own workers and writes their outputs at the end.
+template <int SLOTS>
 __global__ void __launch_bounds__(32) select_first_n_kernel(const float* __restrict__ arrival,
                                                             const int32_t* __restrict__ tags,
                                                             int32_t t, int32_t N, int32_t W,
                                                             uint8_t* __restrict__ mask,
                                                             int32_t* __restrict__ order,
                                                             int32_t* __restrict__ info) {
-  __shared__ float s_arrival[SGDB_MAX_WORKERS];
-  __shared__ uint8_t s_valid[SGDB_MAX_WORKERS];
   const unsigned kAll = 0xffffffffu;
   const int lane = threadIdx.x;
-  const int slots = (W + 31) / 32;
 
+  float a[SLOTS];
+  bool valid[SLOTS];
+  unsigned valid_votes[SLOTS];  // warp-uniform: bit l = worker k*32 + l is valid
   int n_valid = 0;
-  for (int k = 0; k < slots; ++k) {
+#pragma unroll
+  for (int k = 0; k < SLOTS; ++k) {
     const int j = k * 32 + lane;
-    float a = 0.0f;
-    bool valid = false;
-    if (j < W) {
-      a = arrival[j];
-      valid = (tags[j] == t) && isfinite(a);
-      s_arrival[j] = a;
-      s_valid[j] = valid ? 1 : 0;
-    }
-    n_valid += __popc(__ballot_sync(kAll, valid));
+    a[k] = j < W ? arrival[j] : 0.0f;
+    const int tg = j < W ? tags[j] : 0;
+    valid[k] = (j < W) && (tg == t) && isfinite(a[k]);
   }
-  __syncwarp();
+#pragma unroll
+  for (int k = 0; k < SLOTS; ++k) {
+    valid_votes[k] = __ballot_sync(kAll, valid[k]);
+    n_valid += __popc(valid_votes[k]);
+  }
   const bool enough = n_valid >= N;
   if (lane == 0) {
     info[0] = n_valid;
@@ -55,26 +61,33 @@ __global__ void __launch_bounds__(32) select_first_n_kernel(const float* __restr
   }
   if (!enough) return;  // mask and order stay as they were
 
-  for (int w = 0; w < W; ++w) {
-    if (!s_valid[w]) {
-      if (lane == 0) mask[w] = 0;
-      continue;
-    }
-    const float aw = s_arrival[w];
-    int rank = 0;
-    for (int k = 0; k < slots; ++k) {
-      const int j = k * 32 + lane;
-      bool before = false;
-      if (j < W && s_valid[j]) {
-        const float aj = s_arrival[j];
-        before = (aj < aw) || (aj == aw && j < w);
+  int my_rank[SLOTS];
+#pragma unroll
+  for (int kw = 0; kw < SLOTS; ++kw) {
+    my_rank[kw] = 0;
+    if (kw * 32 >= W) continue;
+#pragma unroll 4
+    for (int l = 0; l < 32; ++l) {
+      const float aw = __shfl_sync(kAll, a[kw], l);
+      if (!((valid_votes[kw] >> l) & 1u)) continue;  // uniform: the candidate is not valid
+      const int w = kw * 32 + l;
+      int rank = 0;
+#pragma unroll
+      for (int k = 0; k < SLOTS; ++k) {
+        const int j = k * 32 + lane;
+        const bool before = valid[k] && ((a[k] < aw) || (a[k] == aw && j < w));
+        rank += __popc(__ballot_sync(kAll, before));
       }
-      rank += __popc(__ballot_sync(kAll, before));
+      if (l == lane) my_rank[kw] = rank;
     }
-    if (lane == 0) {
-      const bool kept = rank < N;
-      mask[w] = kept ? 1 : 0;
-      if (kept) order[rank] = w;
+  }
+#pragma unroll
+  for (int k = 0; k < SLOTS; ++k) {
+    const int j = k * 32 + lane;
+    if (j < W) {
+      const bool kept = valid[k] && my_rank[k] < N;
+      mask[j] = kept ? 1 : 0;
+      if (kept) order[my_rank[k]] = j;
     }
   }
 }

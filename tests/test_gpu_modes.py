@@ -55,6 +55,8 @@ def _make_model(dev, lengths, W, kind, dtype, seed, packed):
 def _regen(segs, scales, seed, t, W, dtype, dev, packed):
     for i, (theta, _, _, grad) in enumerate(segs):
         L = theta.numel()
+        if L == 0:
+            continue
         if packed:
             wl.grad_matrix(seed + i, t, W, L, scales, dtype, dev, out=grad)
         else:
