@@ -302,10 +302,10 @@ def finish(args, cfg, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clock
             "pct_of_nominal_8tbs": 100.0 * total_gbs_per_gpu / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": total_gbs_per_gpu, "peak": peak, "unit": "GB/s",
                          "frac": total_gbs_per_gpu / peak, "traffic": traffic, "peak_source": peak_kind,
-                         "kernel": "stream_rows_kernel<float, rmsprop> (duration = whole step, including the one-warp select launch)",
+                         "kernel": "stream_rows_kernel<float, rmsprop> (the step is this one launch)",
                          "algorithmic_bytes_per_launch": total_bytes},
             "e2e": e2e,
-            "gpu_launches": 2 * args.steps,
+            "gpu_launches": args.steps,  # one fused launch per step (selection is the kernel's prologue)
             "clocks": clocks.summary(),
             "cpu_baseline": cpu,
         }

@@ -153,8 +153,9 @@ sgdb_status_t sgdb_update(float *d_theta, float *d_state0, float *d_state1, cons
 
 /*
  * sgdb_step -- one whole iteration of Algorithm 4's loop body: select,
- * aggregate and update, with the mean never written to memory.  Arguments as in
- * the three calls above; d_mask, d_order and d_info are outputs here.
+ * aggregate and update, in a single kernel launch; the mean is never written to
+ * memory.  Arguments as in the three calls above; d_mask, d_order and d_info are
+ * outputs here.
  */
 sgdb_status_t sgdb_step(const void *d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld,
                         const float *d_arrival, const int32_t *d_tags, int32_t t, int32_t N,

@@ -19,8 +19,14 @@ constexpr int kMaxDevices = 64;
 
 // Launch shape of the row-streaming kernel: 256 consumer threads + one producer warp,
 // CH 16-byte chunks per thread and row, so a ring slot holds 8 KiB (f32) / 8 KiB (bf16).
-constexpr int kNT = 256;
-constexpr int kCH = 2;
+#ifndef SGDB_NT
+#define SGDB_NT 256
+#endif
+#ifndef SGDB_CH
+#define SGDB_CH 2
+#endif
+constexpr int kNT = SGDB_NT;
+constexpr int kCH = SGDB_CH;
 constexpr int kStageBytes = kNT * kCH * 16;
 constexpr int kDefaultStages = 6;
 constexpr int kDefaultCtasPerSm = 2;
@@ -132,7 +138,8 @@ sgdb_status_t launch_stream_t(const StreamParams& p_in, long long total_tiles_hi
   auto kernel = stream_rows_kernel<GT, EP, kNT, kCH>;
 
   // shared memory: ring + 2 barriers per slot + order[N] + tile prefix[S + 1]
-  const size_t fixed = static_cast<size_t>((p.N + 3) & ~3) * 4 + (p.table ? (static_cast<size_t>(p.S) + 1) * 4 : 0) + 16;
+  const size_t fixed = static_cast<size_t>((p.N + 3) & ~3) * 4 + (p.table ? (static_cast<size_t>(p.S) + 1) * 4 : 0) +
+                       (p.arrival ? static_cast<size_t>(p.W) * 4 : 0) + 16;
   int ctas_per_sm = g_ctas_per_sm;
   int stages = g_stages;
   const size_t per_sm_budget = static_cast<size_t>(dev->max_smem_optin);
@@ -147,7 +154,12 @@ sgdb_status_t launch_stream_t(const StreamParams& p_in, long long total_tiles_hi
       cudaSuccess)
     return launch_status();
   long long grid = static_cast<long long>(dev->sms) * ctas_per_sm;
-  if (total_tiles_hint > 0 && total_tiles_hint < grid) grid = total_tiles_hint;
+  if (p.table == nullptr) {
+    const long long tile = static_cast<long long>(kNT) * kCH * GradTraits<GT>::kVec;
+    p.total_tiles = static_cast<int>((p.flat.len + tile - 1) / tile);
+    if (p.total_tiles < grid) grid = p.total_tiles;
+  }
+  (void)total_tiles_hint;
   if (grid < 1) grid = 1;
   kernel<<<static_cast<unsigned>(grid), kNT + 32, smem, stream>>>(p);
   return launch_status();
@@ -178,14 +190,23 @@ long long tiles_of(int dt, long long len) {
 sgdb_status_t launch_select(const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t N, int32_t b,
                             uint8_t* d_mask, int32_t* d_order, int32_t* d_info, cudaStream_t stream) {
   const int W = N + b;
-  // the kernel is instantiated for 1, 2, 4, ... workers per lane; take the smallest that holds W
-  if (W <= 32) select_first_n_kernel<1><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
-  else if (W <= 64) select_first_n_kernel<2><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
-  else if (W <= 128) select_first_n_kernel<4><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
-  else if (W <= 256) select_first_n_kernel<8><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
-  else if (W <= 512) select_first_n_kernel<16><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
-  else select_first_n_kernel<32><<<1, 32, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
+  const int threads = (W + 31) & ~31;  // one thread per worker
+  select_first_n_kernel<<<1, threads, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
   return launch_status();
+}
+
+void set_in_kernel_selection(StreamParams* p, const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t W,
+                             uint8_t* d_mask, int32_t* d_order, int32_t* d_info) {
+  p->order = nullptr;
+  p->info = nullptr;
+  p->status_out = d_info + 1;
+  p->arrival = d_arrival;
+  p->tags = d_tags;
+  p->t = t;
+  p->W = W;
+  p->mask_out = d_mask;
+  p->order_out = d_order;
+  p->info_out = d_info;
 }
 
 sgdb_status_t check_flat(const void* grad, int dt, int64_t P, int64_t ld, int32_t N) {
@@ -273,8 +294,7 @@ sgdb_status_t sgdb_step(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t 
   if (d_theta == nullptr || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
     return SGDB_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  st = launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
-  if (st != SGDB_OK || P == 0) return st;
+  if (P == 0) return launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
   StreamParams p{};
   p.table = nullptr;
   p.flat.theta = d_theta;
@@ -285,11 +305,9 @@ sgdb_status_t sgdb_step(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t 
   p.flat.len = P;
   p.S = 1;
   p.N = N;
-  p.order = d_order;
-  p.info = d_info;
-  p.status_out = d_info + 1;
+  set_in_kernel_selection(&p, d_arrival, d_tags, t, N + b, d_mask, d_order, d_info);
   p.h = h;
-  return launch_stream(dt, ep, p, tiles_of(dt, P), s);
+  return launch_stream(dt, ep, p, tiles_of(dt, P), s);  // one launch: selection is the kernel's prologue
 }
 
 sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, sgdb_dtype_t dt,
@@ -308,15 +326,12 @@ sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, s
   st = prepare_rule(opt, &dummy, &dummy, &h, &ep);
   if (st != SGDB_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  st = launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
-  if (st != SGDB_OK || S == 0) return st;
+  if (S == 0) return launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
   StreamParams p{};
   p.table = d_segments;
   p.S = S;
   p.N = N;
-  p.order = d_order;
-  p.info = d_info;
-  p.status_out = d_info + 1;
+  set_in_kernel_selection(&p, d_arrival, d_tags, t, N + b, d_mask, d_order, d_info);
   p.h = h;
   return launch_stream(dt, ep, p, 0, s);
 }

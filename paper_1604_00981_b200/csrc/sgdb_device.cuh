@@ -56,17 +56,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return done != 0;
 }
 
-// Every wait on a barrier is bounded.  In a correct run a phase completes within
-// microseconds; the limit only exists so that a broken pipeline ends the kernel with
-// an error status instead of hanging the device.  `abort_flag` (shared memory) lets
-// one thread's time-out end every other thread's wait quickly.
-constexpr uint32_t kSpinLimit = 1u << 22;
+// Every wait on a barrier is bounded by wall time.  In a correct run a phase completes
+// within microseconds; the limit only exists so that a broken pipeline ends the kernel
+// with an error status instead of hanging the device.  `abort_flag` (shared memory)
+// lets one thread's time-out end every other thread's wait quickly.
+constexpr unsigned long long kWaitLimitNs = 2000ull * 1000 * 1000;  // 2 s
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+  const unsigned long long deadline = global_timer_ns() + kWaitLimitNs;
+  for (uint32_t spin = 0;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 63u) == 63u && *abort_flag != 0) return false;
+    if ((spin & 15u) == 15u) {
+      if (*abort_flag != 0) return false;
+      if (global_timer_ns() > deadline) break;
+    }
   }
   *abort_flag = 1;
   return false;

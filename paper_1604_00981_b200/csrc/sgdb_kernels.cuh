@@ -17,79 +17,82 @@ namespace sgdb {
 
 // ====================================================================== selection
 //
-// One warp.  Worker j is valid when tag[j] == t and its arrival time is finite.
-// The rank of a valid worker w is the number of valid workers that arrive before it,
-// where "before" compares (arrival time, worker id).  Workers of rank < N are kept;
+// Worker j is valid when tag[j] == t and its arrival time is finite.  The rank of a
+// valid worker w is the number of valid workers that arrive before it, where
+// "before" compares (arrival time, worker id).  Workers of rank < N are kept;
 // order[rank] = w puts them in arrival sequence.
 //
-// Lane l keeps workers l, l + 32, ... (SLOTS of them) in registers.  Candidates are
-// taken one at a time: the owning lane broadcasts its key with __shfl_sync, every
-// lane tests its own workers against it, and the votes are counted with
-// __ballot_sync / __popc.  All loops over slots are unrolled, so the single warp has
-// enough independent work in flight to hide its own latencies.  Each lane remembers
-// the ranks of its own workers and writes their outputs at the end.
-template <int SLOTS>
-__global__ void __launch_bounds__(32) select_first_n_kernel(const float* __restrict__ arrival,
-                                                            const int32_t* __restrict__ tags,
-                                                            int32_t t, int32_t N, int32_t W,
-                                                            uint8_t* __restrict__ mask,
-                                                            int32_t* __restrict__ order,
-                                                            int32_t* __restrict__ info) {
-  const unsigned kAll = 0xffffffffu;
-  const int lane = threadIdx.x;
-
-  float a[SLOTS];
-  bool valid[SLOTS];
-  unsigned valid_votes[SLOTS];  // warp-uniform: bit l = worker k*32 + l is valid
-  int n_valid = 0;
-#pragma unroll
-  for (int k = 0; k < SLOTS; ++k) {
-    const int j = k * 32 + lane;
-    a[k] = j < W ? arrival[j] : 0.0f;
-    const int tg = j < W ? tags[j] : 0;
-    valid[k] = (j < W) && (tg == t) && isfinite(a[k]);
+// block_select is called by every thread of a block.  Thread i owns workers i,
+// i + blockDim.x, ...; keys of valid workers go to shared memory (NaN for the others,
+// which never compares as "before"), the valid ones are counted with
+// __ballot_sync / __popc, and each thread ranks its own workers with one pass over
+// the keys.  A one-warp version that ranked by ballots over register-resident keys
+// measured 20 us for W = 100 on a B200 (one warp cannot hide its own latencies);
+// this form takes about as long as the load of its inputs.
+//
+//   s_key   [W] floats of shared memory, s_order [N] ints, s_count one int
+//   g_mask / g_order / g_info: global outputs, written only when `writer`
+// Returns true when at least N workers are valid; s_order is then filled.  When it
+// returns false nothing but g_info has been written.
+__device__ __forceinline__ bool block_select(const float* __restrict__ arrival,
+                                             const int32_t* __restrict__ tags, int32_t t, int32_t N,
+                                             int32_t W, float* s_key, int* s_order, int* s_count,
+                                             bool writer, uint8_t* __restrict__ g_mask,
+                                             int32_t* __restrict__ g_order,
+                                             int32_t* __restrict__ g_info) {
+  const int tid = threadIdx.x;
+  const int nthreads = blockDim.x;
+  if (tid == 0) *s_count = 0;
+  __syncthreads();
+  const int w_end = (W + 31) & ~31;  // whole warps take part in every ballot
+  for (int w = tid; w < w_end; w += nthreads) {
+    bool valid = false;
+    float a = 0.0f;
+    if (w < W) {
+      a = arrival[w];
+      valid = (tags[w] == t) && isfinite(a);
+      s_key[w] = valid ? a : __int_as_float(0x7fc00000);
+    }
+    const unsigned votes = __ballot_sync(0xffffffffu, valid);
+    if ((tid & 31) == 0 && votes != 0) atomicAdd(s_count, __popc(votes));
   }
-#pragma unroll
-  for (int k = 0; k < SLOTS; ++k) {
-    valid_votes[k] = __ballot_sync(kAll, valid[k]);
-    n_valid += __popc(valid_votes[k]);
-  }
+  __syncthreads();
+  const int n_valid = *s_count;
   const bool enough = n_valid >= N;
-  if (lane == 0) {
-    info[0] = n_valid;
-    info[1] = enough ? SGDB_OK : SGDB_ERR_INSUFFICIENT;
+  if (writer && tid == 0) {
+    g_info[0] = n_valid;
+    g_info[1] = enough ? SGDB_OK : SGDB_ERR_INSUFFICIENT;
   }
-  if (!enough) return;  // mask and order stay as they were
+  if (!enough) return false;
+  for (int w = tid; w < W; w += nthreads) {
+    const float a = s_key[w];
+    int rank = 0;
+#pragma unroll 8
+    for (int j = 0; j < W; ++j) {
+      const float aj = s_key[j];
+      rank += ((aj < a) || (aj == a && j < w)) ? 1 : 0;
+    }
+    const bool kept = (a == a) && rank < N;  // a != a: not valid
+    if (kept) s_order[rank] = w;
+    if (writer) {
+      g_mask[w] = kept ? 1 : 0;
+      if (kept) g_order[rank] = w;
+    }
+  }
+  __syncthreads();
+  return true;
+}
 
-  int my_rank[SLOTS];
-#pragma unroll
-  for (int kw = 0; kw < SLOTS; ++kw) {
-    my_rank[kw] = 0;
-    if (kw * 32 >= W) continue;
-#pragma unroll 4
-    for (int l = 0; l < 32; ++l) {
-      const float aw = __shfl_sync(kAll, a[kw], l);
-      if (!((valid_votes[kw] >> l) & 1u)) continue;  // uniform: the candidate is not valid
-      const int w = kw * 32 + l;
-      int rank = 0;
-#pragma unroll
-      for (int k = 0; k < SLOTS; ++k) {
-        const int j = k * 32 + lane;
-        const bool before = valid[k] && ((a[k] < aw) || (a[k] == aw && j < w));
-        rank += __popc(__ballot_sync(kAll, before));
-      }
-      if (l == lane) my_rank[kw] = rank;
-    }
-  }
-#pragma unroll
-  for (int k = 0; k < SLOTS; ++k) {
-    const int j = k * 32 + lane;
-    if (j < W) {
-      const bool kept = valid[k] && my_rank[k] < N;
-      mask[j] = kept ? 1 : 0;
-      if (kept) order[my_rank[k]] = j;
-    }
-  }
+__global__ void __launch_bounds__(1024) select_first_n_kernel(const float* __restrict__ arrival,
+                                                              const int32_t* __restrict__ tags,
+                                                              int32_t t, int32_t N, int32_t W,
+                                                              uint8_t* __restrict__ mask,
+                                                              int32_t* __restrict__ order,
+                                                              int32_t* __restrict__ info) {
+  __shared__ float s_key[SGDB_MAX_WORKERS];
+  __shared__ int s_order[SGDB_MAX_WORKERS];
+  __shared__ int s_count;
+  block_select(arrival, tags, t, N, W, s_key, s_order, &s_count, true, mask, order, info);
 }
 
 // ====================================================================== row streaming
@@ -113,11 +116,22 @@ struct StreamParams {
   const sgdb_segment_t* table;  // device segment table, or nullptr: use `flat`
   sgdb_segment_t flat;          // with EP_MEAN, flat.theta is where the mean goes
   int S;                        // entries in `table`
+  int total_tiles;              // flat case: number of TILE-wide tiles (tables: counted in the kernel)
   int N;                        // rows to add
   int stages;                   // ring depth
-  const int32_t* order;         // [N] row ids in summation order
+  const int32_t* order;         // [N] row ids in summation order (when the selection is given)
   const int32_t* info;          // optional [2]; info[1] != SGDB_OK: do nothing
   int32_t* status_out;          // optional: receives SGDB_ERR_TIMEOUT if a wait runs out
+  // When `arrival` is not null the kernel takes the selection itself: every block
+  // ranks the W workers in its prologue (the same deterministic result in each) and
+  // block 0 writes mask_out, order_out and info_out.
+  const float* arrival;
+  const int32_t* tags;
+  int32_t t;
+  int32_t W;
+  uint8_t* mask_out;
+  int32_t* order_out;
+  int32_t* info_out;
   Hyper h;
 };
 
@@ -178,8 +192,7 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
 
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ int s_abort;
-
-  if (p.info != nullptr && p.info[1] != SGDB_OK) return;  // e.g. fewer than N current gradients
+  __shared__ int s_count;
 
   const int tid = threadIdx.x;
   const int lane = tid & 31;
@@ -189,8 +202,17 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
   uint64_t* empty_bar = full_bar + stages;
   int* order_s = reinterpret_cast<int*>(empty_bar + stages);
   int* prefix_s = order_s + ((N + 3) & ~3);
+  float* key_s = reinterpret_cast<float*>(prefix_s + (p.table != nullptr ? p.S + 1 : 0));
 
-  for (int i = tid; i < N; i += NT + 32) order_s[i] = p.order[i];
+  if (p.arrival != nullptr) {
+    // fewer than N current gradients: the iteration cannot complete, nothing is touched
+    if (!block_select(p.arrival, p.tags, p.t, N, p.W, key_s, order_s, &s_count, blockIdx.x == 0,
+                      p.mask_out, p.order_out, p.info_out))
+      return;
+  } else {
+    if (p.info != nullptr && p.info[1] != SGDB_OK) return;
+    for (int i = tid; i < N; i += NT + 32) order_s[i] = p.order[i];
+  }
   if (tid == 0) {
     s_abort = 0;
     for (int s = 0; s < stages; ++s) {
@@ -224,8 +246,7 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
     }
   }
   __syncthreads();
-  const int total_tiles =
-      p.table != nullptr ? prefix_s[p.S] : static_cast<int>((p.flat.len + TILE - 1) / TILE);
+  const int total_tiles = p.table != nullptr ? prefix_s[p.S] : p.total_tiles;
   const uint32_t ring_addr = smem_addr(smem);
   const uint32_t full_addr = smem_addr(full_bar);
   const uint32_t empty_addr = smem_addr(empty_bar);
