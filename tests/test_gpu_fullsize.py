@@ -1,0 +1,191 @@
+"""Parity at the full sizes of the five workloads, in the launch configuration the benchmark times.
+
+The oracle cannot chew through 10-40 GB in seconds, but the path is separable by column: the oracle
+runs on a sample of columns (random ones, the first and last, and tile borders) cut out of the very
+matrices the GPU consumed, and the GPU's results are compared at those columns.  Whole-vector
+properties that hold at any size are checked as well (bitwise agreement between the fused step and
+the other entry points, untouched padding, finite results).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import (TOL_BF16, TOL_F32, gpu_opt, gpu_state, oracle_opt, oracle_state, rel_err,
+                     selection_buffers, step_inputs, to_dev)
+from paper_1604_00981_b200 import workload as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sgdb(cuda_device):
+    from paper_1604_00981_b200 import binding
+
+    return binding
+
+
+def _need_memory(dev, gigabytes):
+    free, _ = torch.cuda.mem_get_info(dev)
+    if free < gigabytes * 1e9:
+        pytest.skip("needs %.0f GB of free device memory" % gigabytes)
+
+
+def _sample_columns(P, rng, n=3000, tile=2048):
+    cols = [rng.integers(0, P, size=min(n, P)), np.arange(min(16, P)), np.arange(max(0, P - 16), P)]
+    for k in rng.integers(1, max(2, P // tile), size=8):
+        cols.append(np.array([k * tile - 1, k * tile, min(P - 1, k * tile + 1)]))
+    cols = np.unique(np.concatenate(cols))
+    return cols[(cols >= 0) & (cols < P)].astype(np.int64)
+
+
+def _flat_trajectory_sampled(sgdb, dev, cfg, T):
+    W, N, P, kind = cfg.W, cfg.N, cfg.P, cfg.opt["kind"]
+    rng = np.random.default_rng(cfg.seed)
+    cols = _sample_columns(P, rng, tile=2048 if cfg.grad_dtype == "f32" else 4096)
+    cols_d = to_dev(cols, dev)
+    scales = wl.worker_scales(cfg.seed, W)
+    theta = wl.theta0(cfg.seed, P, dev)
+    s0, s1 = gpu_state(kind, P, dev)
+    th_o = theta[cols_d].cpu().numpy().astype(np.float64)
+    s0_o, s1_o = oracle_state(kind, len(cols))
+    mask, order, info = selection_buffers(W, N, dev)
+    grad = None
+    for t in range(T):
+        grad = wl.grad_matrix(cfg.seed, t, W, P, scales, cfg.grad_dtype, dev, out=grad)
+        arrival, tags = step_inputs(cfg.seed, t, W, N)
+        sgdb.sgdb_step(grad, P, to_dev(arrival, dev), to_dev(tags, dev), t, N, cfg.b, theta, s0, s1,
+                       gpu_opt(cfg.opt, t + 1), mask, order, info)
+        sample = wl.as_oracle_array(grad.index_select(1, cols_d))
+        rc, mask_o, order_o, n_valid = oracle.step(sample, len(cols), arrival, tags, t, N, cfg.b, th_o, s0_o, s1_o,
+                                                   oracle_opt(cfg.opt, t + 1))
+        assert rc == oracle.OK and info.cpu().tolist() == [n_valid, 0]
+        assert mask.cpu().numpy().tolist() == mask_o.tolist()
+        assert order.cpu().numpy().tolist() == order_o.tolist()
+    tol = TOL_F32 if cfg.grad_dtype == "f32" else TOL_BF16
+    assert rel_err(theta[cols_d].cpu().numpy(), th_o) < tol
+    assert rel_err(s0[cols_d].cpu().numpy(), s0_o) < tol
+    assert rel_err(s1[cols_d].cpu().numpy(), s1_o) < tol
+    assert bool(torch.isfinite(theta).all())
+    return grad, theta, s0, s1, arrival, tags, T - 1
+
+
+def test_config1_full_size(sgdb, cuda_device):
+    """P = 23.8 M fp32, W = 100 (N = 96, b = 4), RMSProp; fused step vs oracle at sampled columns, then the
+    separate select / aggregate / update calls against the fused step on the whole vector."""
+    _need_memory(cuda_device, 12)
+    dev, cfg = cuda_device, wl.CONFIGS[1]
+    grad, theta, s0, s1, arrival, tags, t = _flat_trajectory_sampled(sgdb, dev, cfg, T=3)
+    W, N, P = cfg.W, cfg.N, cfg.P
+    th_f, s0_f, s1_f = theta.clone(), s0.clone(), s1.clone()
+    mask, order, info = selection_buffers(W, N, dev)
+    a_d, t_d = to_dev(arrival, dev), to_dev(tags, dev)
+    opt = gpu_opt(cfg.opt, t + 2)
+    sgdb.sgdb_step(grad, P, a_d, t_d, t, N, cfg.b, th_f, s0_f, s1_f, opt, mask, order, info)
+    mean = torch.empty(P, device=dev)
+    mask2, order2, info2 = selection_buffers(W, N, dev)
+    sgdb.sgdb_select(a_d, t_d, t, N, cfg.b, mask2, order2, info2)
+    sgdb.sgdb_aggregate(grad, P, N, order2, info2, mean)
+    sgdb.sgdb_update(theta, s0, s1, mean, opt, info2)
+    assert torch.equal(order, order2) and torch.equal(mask, mask2)
+    assert torch.equal(theta, th_f) and torch.equal(s0, s0_f) and torch.equal(s1, s1_f)
+
+
+def test_config3_full_size(sgdb, cuda_device):
+    """P = 100 M, W = 208 (N = 200, b = 8), bf16 rows (41.6 GB), Adam."""
+    _need_memory(cuda_device, 48)
+    _flat_trajectory_sampled(sgdb, cuda_device, wl.CONFIGS[3], T=2)
+
+
+def test_config2_full_size_segmented(sgdb, cuda_device):
+    """300 tensors with log-uniform lengths in [64, 2^21], W = 54 (N = 50, b = 4), momentum SGD:
+    one launch over the device table vs the oracle (small tensors whole, large ones at sampled columns)
+    and vs one fused launch per tensor (bitwise)."""
+    _need_memory(cuda_device, 20)
+    dev, cfg = cuda_device, wl.CONFIGS[2]
+    W, N, kind = cfg.W, cfg.N, cfg.opt["kind"]
+    lengths = wl.segment_lengths(cfg.seed, cfg.segments)
+    rng = np.random.default_rng(cfg.seed)
+    scales = wl.worker_scales(cfg.seed, W)
+    segs, samples = [], []
+    for i, L in enumerate(int(x) for x in lengths):
+        ld = (L + 3) // 4 * 4
+        theta = wl.theta0(cfg.seed + i, L, dev)
+        grad = wl.grad_matrix(cfg.seed + i, 0, W, L, scales, "f32", dev, ld=ld)
+        segs.append((theta, torch.zeros(L, device=dev), None, grad))
+        cols = np.arange(L) if L <= 4096 else _sample_columns(L, rng, n=256)
+        samples.append(cols)
+    twins = [(s[0].clone(), s[1].clone()) for s in segs]
+    table = sgdb.make_segment_table(segs, dev)
+    th_o = [segs[i][0][to_dev(samples[i], dev)].cpu().numpy().astype(np.float64) for i in range(len(segs))]
+    v_o = [np.zeros(len(c)) for c in samples]
+    mask, order, info = selection_buffers(W, N, dev)
+    mask2, order2, info2 = selection_buffers(W, N, dev)
+    for t in range(2):
+        if t:
+            for i, (theta, _, _, grad) in enumerate(segs):
+                wl.grad_matrix(cfg.seed + i, t, W, theta.numel(), scales, "f32", dev, ld=grad.stride(0), out=grad)
+        arrival, tags = step_inputs(cfg.seed, t, W, N)
+        a_d, t_d = to_dev(arrival, dev), to_dev(tags, dev)
+        sgdb.sgdb_step_segmented(table, len(segs), torch.float32, a_d, t_d, t, N, cfg.b, gpu_opt(cfg.opt, t + 1),
+                                 mask, order, info)
+        rc, mask_o, order_o, n_valid = oracle.select(arrival, tags, t, N, cfg.b)
+        assert rc == oracle.OK and info.cpu().tolist() == [n_valid, 0]
+        assert order.cpu().numpy().tolist() == order_o.tolist()
+        for i, (theta, v, _, grad) in enumerate(segs):
+            cols_d = to_dev(samples[i], dev)
+            sample = wl.as_oracle_array(grad.index_select(1, cols_d))
+            mean = oracle.aggregate(sample, len(samples[i]), order_o)
+            oracle.update(th_o[i], v_o[i], None, mean, oracle_opt(cfg.opt, t + 1))
+            if i % 10 == 0:  # one launch per tensor, every tenth tensor
+                sgdb.sgdb_step(grad, theta.numel(), a_d, t_d, t, N, cfg.b, twins[i][0], twins[i][1], None,
+                               gpu_opt(cfg.opt, t + 1), mask2, order2, info2, ld=grad.stride(0))
+    got = np.concatenate([segs[i][0][to_dev(samples[i], dev)].cpu().numpy() for i in range(len(segs))])
+    got_v = np.concatenate([segs[i][1][to_dev(samples[i], dev)].cpu().numpy() for i in range(len(segs))])
+    assert rel_err(got, np.concatenate(th_o)) < TOL_F32
+    assert rel_err(got_v, np.concatenate(v_o)) < TOL_F32
+    for i in range(0, len(segs), 10):
+        assert torch.equal(segs[i][0], twins[i][0]) and torch.equal(segs[i][1], twins[i][1]), i
+
+
+@pytest.mark.parametrize("b", [0, 2, 4, 8])
+def test_config4_full_size_accumulate_on_arrival(sgdb, cuda_device, b):
+    """P = 23.8 M fp32, N = 96, b swept: one iteration delivered row by row in arrival sequence;
+    outcomes replayed by the oracle's arrival-by-arrival server, parameters compared at sampled columns
+    with the oracle and on the whole vector with the fused step (bitwise)."""
+    _need_memory(cuda_device, 14)
+    dev, cfg = cuda_device, wl.CONFIGS[4]
+    N, P, kind = cfg.N, cfg.P, cfg.opt["kind"]
+    W = N + b
+    seed = cfg.seed + b
+    rng = np.random.default_rng(seed)
+    cols = _sample_columns(P, rng)
+    cols_d = to_dev(cols, dev)
+    grad = wl.grad_matrix(seed, 0, W, P, wl.worker_scales(seed, W), "f32", dev)
+    arrival, tags = step_inputs(seed, 0, W, N)
+    theta = wl.theta0(seed, P, dev)
+    theta_f = theta.clone()
+    s0, s1 = gpu_state(kind, P, dev)
+    sf = gpu_state(kind, P, dev)
+    acc = torch.empty(P, device=dev)
+    counter = torch.zeros(4, dtype=torch.int32, device=dev)
+    info = torch.zeros(2, dtype=torch.int32, device=dev)
+    th_o = theta[cols_d].cpu().numpy().astype(np.float64)
+    s0_o, s1_o = oracle_state(kind, len(cols))
+    acc_o, state_o = np.zeros(len(cols)), oracle.new_server_state()
+    sample = wl.as_oracle_array(grad.index_select(1, cols_d))
+    outcomes = []
+    for w in wl.delivery_sequence(arrival):
+        sgdb.sgdb_accumulate_arrival(grad[w], int(tags[w]), 0, N, acc, counter, theta, s0, s1, gpu_opt(cfg.opt), info)
+        want = oracle.accumulate_arrival(sample[w], int(tags[w]), 0, N, acc_o, state_o, th_o, s0_o, s1_o,
+                                         oracle_opt(cfg.opt))
+        assert info.cpu().tolist()[0] == want
+        outcomes.append(want)
+    assert outcomes.count(2) == 1 and outcomes.count(1) == N - 1
+    assert counter.cpu().tolist() == [0, len(outcomes), 0, 1]
+    assert rel_err(theta[cols_d].cpu().numpy(), th_o) < TOL_F32
+    assert rel_err(s0[cols_d].cpu().numpy(), s0_o) < TOL_F32
+    mask, order, finfo = selection_buffers(W, N, dev)
+    sgdb.sgdb_step(grad, P, to_dev(arrival, dev), to_dev(tags, dev), 0, N, b, theta_f, sf[0], sf[1], gpu_opt(cfg.opt),
+                   mask, order, finfo)
+    assert torch.equal(theta, theta_f) and torch.equal(s0, sf[0]) and torch.equal(s1, sf[1])
