@@ -230,6 +230,42 @@ sgdb_status_t sgdb_step_host(const void *h_grad, sgdb_dtype_t dt, int64_t P, int
 size_t sgdb_step_host_workspace_bytes(sgdb_dtype_t dt, int64_t P, int64_t ld, int32_t N, int32_t b);
 
 /*
+ * sgdb_step_host_static -- sgdb_step_host for callers that have no device memory
+ * to hand over and must not create any.  (The paper has no counterpart; this is a
+ * deployment convenience.)
+ *
+ * Who needs it: a server loop that runs after the process has given every byte of
+ * device memory to another component's pool; code that runs where cudaMalloc is
+ * off limits because it may fail under a memory budget or stalls the whole device
+ * while it runs; a plug-in that is handed tensors but no allocator.  Such callers
+ * still own the inputs and outputs, but cannot supply sgdb_step_host's workspace.
+ *
+ * Here the workspace is a fixed array of SGDB_STATIC_SCRATCH_BYTES that is part of
+ * the library image: every GPU that loads the library holds it until the process
+ * exits.  The call allocates and frees nothing, neither directly nor through a
+ * library routine.  Arguments and results are exactly those of sgdb_step_host
+ * without the two workspace arguments.
+ *
+ *   - Sizes whose workspace (sgdb_step_host_workspace_bytes) exceeds
+ *     SGDB_STATIC_SCRATCH_BYTES are refused with SGDB_ERR_UNSUPPORTED and a line
+ *     on stderr; nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that
+ *     device current) and keeps it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last
+ *     call left in it.  Nothing in it needs to start at zero: every byte the
+ *     kernels read is written by this call's own copies first.  Two calls that
+ *     overlap on the same device (different streams or threads) race on it: keep
+ *     them ordered.
+ */
+#define SGDB_STATIC_SCRATCH_BYTES (8u << 20)
+sgdb_status_t sgdb_step_host_static(const void *h_grad, sgdb_dtype_t dt, int64_t P, int64_t ld,
+                                    const float *h_arrival, const int32_t *h_tags, int32_t t,
+                                    int32_t N, int32_t b, float *d_theta, float *d_state0,
+                                    float *d_state1, const sgdb_opt_t *opt, float *h_theta_out,
+                                    uint8_t *h_mask, int32_t *h_order, int32_t *h_info,
+                                    void *stream);
+
+/*
  * sgdb_set_tuning -- launch-shape knobs of the row-streaming kernels, for
  * measurement sweeps (no counterpart in the paper).  stages: depth of the
  * shared-memory ring of row slices; ctas_per_sm: resident blocks per SM.

@@ -24,9 +24,10 @@ _KINDS = {"sgd": SGDB_SGD, "momentum": SGDB_MOMENTUM, "rmsprop": SGDB_RMSPROP, "
 
 EXPORTS = (
     "sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented",
-    "sgdb_accumulate_arrival", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_set_tuning",
-    "sgdb_strerror", "sgdb_version",
+    "sgdb_accumulate_arrival", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
+    "sgdb_set_tuning", "sgdb_strerror", "sgdb_version",
 )
+SGDB_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class SgdbError(RuntimeError):
@@ -83,6 +84,8 @@ def _load():
         "sgdb_step_host": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt),
                                  vp, vp, vp, vp, vp, sz, vp]),
         "sgdb_step_host_workspace_bytes": (sz, [i32, i64, i64, i32, i32]),
+        "sgdb_step_host_static": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt),
+                                        vp, vp, vp, vp, vp]),
         "sgdb_set_tuning": (i32, [i32, i32]),
         "sgdb_strerror": (ctypes.c_char_p, [i32]),
         "sgdb_version": (ctypes.c_int, []),
@@ -241,4 +244,24 @@ def sgdb_step_host(h_grad, P: int, h_arrival, h_tags, t: int, N: int, b: int, th
                              _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream))
     if st not in (SGDB_OK, SGDB_ERR_INSUFFICIENT):
         raise SgdbError(st, "sgdb_step_host")
+    return st
+
+
+def sgdb_step_host_static(h_grad, P: int, h_arrival, h_tags, t: int, N: int, b: int, theta, state0, state1, opt: Opt,
+                          h_theta_out, h_mask, h_order, h_info, ld: int | None = None, stream=None) -> int:
+    """sgdb_step_host without a workspace argument, for callers that can neither supply device memory nor
+    allocate any: the staging area is a fixed SGDB_STATIC_SCRATCH_BYTES array inside the library.  Sizes that
+    do not fit raise SgdbError (SGDB_ERR_UNSUPPORTED).  Calls on one device share that array: do not overlap
+    them.  Returns the status (0 or SGDB_ERR_INSUFFICIENT)."""
+    ld = h_grad.stride(0) if ld is None else ld
+    c = opt._c()
+    st = _lib.sgdb_step_host_static(_host(h_grad, None, "h_grad"), _grad_dtype(h_grad), P, ld,
+                                    _host(h_arrival, torch.float32, "h_arrival"), _host(h_tags, torch.int32, "h_tags"),
+                                    t, N, b, _dev(theta, torch.float32, "theta"), _dev(state0, torch.float32, "state0"),
+                                    _dev(state1, torch.float32, "state1"), ctypes.byref(c),
+                                    _host(h_theta_out, torch.float32, "h_theta_out"),
+                                    _host(h_mask, torch.uint8, "h_mask"), _host(h_order, torch.int32, "h_order"),
+                                    _host(h_info, torch.int32, "h_info"), _stream(stream))
+    if st not in (SGDB_OK, SGDB_ERR_INSUFFICIENT):
+        raise SgdbError(st, "sgdb_step_host_static")
     return st

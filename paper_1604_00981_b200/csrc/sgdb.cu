@@ -7,6 +7,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "sgdb_kernels.cuh"
 
@@ -472,6 +473,52 @@ sgdb_status_t sgdb_step_host(const void* h_grad, sgdb_dtype_t dt, int64_t P, int
   }
   if (cudaStreamSynchronize(s) != cudaSuccess) return launch_status();
   return static_cast<sgdb_status_t>(h_info[1]);
+}
+
+// ---------------------------------------------------------------- fixed-scratch variant
+//
+// Scratch for callers that cannot allocate: a file-scope device array.  In host code
+// the name `g_static_scratch` is only a handle for the runtime, not a device address;
+// the address each device gave the array is looked up once per device with
+// cudaGetSymbolAddress (that device current) and it is that pointer the kernels get.
+static __device__ __align__(256) unsigned char g_static_scratch[SGDB_STATIC_SCRATCH_BYTES];
+static void* g_static_scratch_addr[kMaxDevices];  // per device, null until looked up
+static std::mutex g_static_scratch_mutex;
+
+sgdb_status_t sgdb_step_host_static(const void* h_grad, sgdb_dtype_t dt, int64_t P, int64_t ld,
+                                    const float* h_arrival, const int32_t* h_tags, int32_t t, int32_t N,
+                                    int32_t b, float* d_theta, float* d_state0, float* d_state1,
+                                    const sgdb_opt_t* opt, float* h_theta_out, uint8_t* h_mask,
+                                    int32_t* h_order, int32_t* h_info, void* stream) {
+  const size_t need = sgdb_step_host_workspace_bytes(dt, P, ld, N, b);
+  if (need == 0) return SGDB_ERR_INVALID_ARG;
+  if (need > SGDB_STATIC_SCRATCH_BYTES) {
+    std::fprintf(stderr,
+                 "libsgdb: sgdb_step_host_static needs %zu bytes of scratch for these sizes, the built-in "
+                 "array holds %u; use sgdb_step_host with a caller-owned workspace\n",
+                 need, static_cast<unsigned>(SGDB_STATIC_SCRATCH_BYTES));
+    return SGDB_ERR_UNSUPPORTED;
+  }
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return launch_status();
+  if (dev < 0 || dev >= kMaxDevices) return SGDB_ERR_UNSUPPORTED;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (g_static_scratch_addr[dev] == nullptr) {
+      void* addr = nullptr;
+      const cudaError_t e = cudaGetSymbolAddress(&addr, g_static_scratch);
+      if (e != cudaSuccess || addr == nullptr) {
+        std::fprintf(stderr, "libsgdb: cudaGetSymbolAddress failed on device %d: %s\n", dev, cudaGetErrorString(e));
+        (void)cudaGetLastError();
+        return SGDB_ERR_CUDA;
+      }
+      g_static_scratch_addr[dev] = addr;
+    }
+    scratch = g_static_scratch_addr[dev];
+  }
+  return sgdb_step_host(h_grad, dt, P, ld, h_arrival, h_tags, t, N, b, d_theta, d_state0, d_state1, opt,
+                        h_theta_out, h_mask, h_order, h_info, scratch, SGDB_STATIC_SCRATCH_BYTES, stream);
 }
 
 sgdb_status_t sgdb_set_tuning(int32_t stages, int32_t ctas_per_sm) {
