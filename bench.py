@@ -168,6 +168,166 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+N_STATE = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2}
+N_SETS = 16  # arrival/tag draws rotate, so the kept set differs from step to step
+
+
+def selection_sets(cfg, dev):
+    arr = [torch.from_numpy(wl.arrivals(cfg.seed, t, cfg.W)).to(dev) for t in range(N_SETS)]
+    tag = [torch.from_numpy(wl.tags(cfg.seed, t, cfg.W, cfg.N) - t).to(dev) for t in range(N_SETS)]  # relative to t = 0
+    return arr, tag
+
+
+def selection_outputs(W, N, dev):
+    return (torch.zeros(W, dtype=torch.uint8, device=dev), torch.zeros(N, dtype=torch.int32, device=dev),
+            torch.zeros(2, dtype=torch.int32, device=dev))
+
+
+def setup_flat(cfg, dev, sgdb, seed):
+    """Workloads with one flat parameter vector (tiny SGD, Inception-sized RMSProp, large bf16 Adam)."""
+    W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
+    scales = wl.worker_scales(cfg.seed, W)
+    grad = wl.grad_matrix(seed, 0, W, P, scales, cfg.grad_dtype, dev)
+    theta = wl.theta0(seed, P, dev)
+    n_state = N_STATE[cfg.opt["kind"]]
+    s0 = torch.zeros(P, device=dev) if n_state >= 1 else None
+    s1 = torch.zeros(P, device=dev) if n_state >= 2 else None
+    mask, order, info = selection_outputs(W, N, dev)
+    arr_d, tag_d = selection_sets(cfg, dev)
+    opt = sgdb.Opt(**cfg.opt)
+
+    def step(i):
+        opt.step = i + 1
+        sgdb.sgdb_step(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, mask, order, info)
+
+    def check():
+        assert info.cpu().tolist()[1] == 0, "a step reported a device-side error"
+        assert bool(torch.isfinite(theta).all())
+
+    grad_bytes = N * P * grad.element_size()
+    state = dict(grad=grad, theta=theta, s0=s0, s1=s1, opt=opt)
+    return dict(step=step, check=check, grad_bytes=grad_bytes, total_bytes=grad_bytes + 2 * (1 + n_state) * P * 4,
+                launches_per_step=1, kernel="stream_rows_kernel<%s, %s> (the step is this one launch)"
+                % (cfg.grad_dtype, cfg.opt["kind"]), state=state, extra={})
+
+
+def setup_segmented(cfg, dev, sgdb, seed):
+    """300 tensors of log-uniform length, one launch over a device-side segment table."""
+    W, N, b = cfg.W, cfg.N, cfg.b
+    scales = wl.worker_scales(cfg.seed, W)
+    lengths = wl.segment_lengths(cfg.seed, cfg.segments)
+    n_state = N_STATE[cfg.opt["kind"]]
+    segs = []
+    for i, L in enumerate(int(x) for x in lengths):
+        ld = (L + 3) // 4 * 4
+        segs.append((wl.theta0(seed + i, L, dev), torch.zeros(L, device=dev) if n_state >= 1 else None,
+                     torch.zeros(L, device=dev) if n_state >= 2 else None,
+                     wl.grad_matrix(seed + i, 0, W, L, scales, cfg.grad_dtype, dev, ld=ld)))
+    table = sgdb.make_segment_table(segs, dev)
+    mask, order, info = selection_outputs(W, N, dev)
+    arr_d, tag_d = selection_sets(cfg, dev)
+    opt = sgdb.Opt(**cfg.opt)
+    P = int(lengths.sum())
+
+    def step(i):
+        opt.step = i + 1
+        sgdb.sgdb_step_segmented(table, len(segs), segs[0][3].dtype, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b,
+                                 opt, mask, order, info)
+
+    def per_tensor_step(i):
+        opt.step = i + 1
+        for theta, s0, s1, grad in segs:
+            sgdb.sgdb_step(grad, theta.numel(), arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt,
+                           mask, order, info, ld=grad.stride(0))
+
+    def check():
+        assert info.cpu().tolist()[1] == 0
+        assert all(bool(torch.isfinite(sg[0]).all()) for sg in segs[:20])
+
+    def extra():
+        ms = time_steps(per_tensor_step, 5, 2)
+        return {"one_launch_per_tensor_ms_per_step": ms, "tensors": len(segs), "total_parameters": P}
+
+    grad_bytes = N * P * segs[0][3].element_size()
+    return dict(step=step, check=check, grad_bytes=grad_bytes, total_bytes=grad_bytes + 2 * (1 + n_state) * P * 4,
+                launches_per_step=1, kernel="stream_rows_kernel<%s, %s> over a %d-entry segment table"
+                % (cfg.grad_dtype, cfg.opt["kind"], len(segs)), state=dict(segs=segs, table=table), extra=extra, P=P)
+
+
+def setup_arrivals(cfg, dev, sgdb, seed):
+    """Accumulate-on-arrival: a step is one whole iteration, W calls in arrival sequence (N accepted, b dropped)."""
+    N, P = cfg.N, cfg.P
+    n_state = N_STATE[cfg.opt["kind"]]
+    b_max = 8
+    scales = wl.worker_scales(cfg.seed, N + b_max)
+    grad = wl.grad_matrix(seed, 0, N + b_max, P, scales, cfg.grad_dtype, dev)
+    theta = wl.theta0(seed, P, dev)
+    s0, s1 = torch.zeros(P, device=dev), torch.zeros(P, device=dev)
+    acc = torch.empty(P, device=dev)
+    counter = torch.zeros(4, dtype=torch.int32, device=dev)
+    info = torch.zeros(2, dtype=torch.int32, device=dev)
+    opt = sgdb.Opt(**cfg.opt)
+    sequences = {bb: [int(w) for w in wl.delivery_sequence(wl.arrivals(cfg.seed + bb, 0, N + bb))] for bb in (0, 2, 4, 8)}
+    iteration = [0]
+
+    def make_step(bb):
+        def step(i):
+            t = iteration[0]
+            opt.step = t + 1
+            for w in sequences[bb]:  # every tag is current; the last bb arrivals come after the update fired
+                sgdb.sgdb_accumulate_arrival(grad[w], t, t, N, acc, counter, theta, s0, s1, opt, info)
+            iteration[0] = t + 1
+        return step
+
+    def check():
+        c = counter.cpu().tolist()
+        assert c[0] == 0 and c[2] == 0 and c[3] == iteration[0], c
+        assert bool(torch.isfinite(theta).all())
+
+    def extra():
+        out = {}
+        for bb in (0, 2, 8):
+            ms = time_steps(make_step(bb), 5, 2)
+            out["b=%d" % bb] = {"ms_per_step": ms, "calls_per_step": N + bb}
+        return {"b_sweep": out, "bytes_per_accepted_arrival": P * 12}
+
+    esize = grad.element_size()
+    grad_bytes = N * P * esize
+    # first accepted row: read row, write acc; middle rows: read row + acc, write acc; N-th: read row + acc + theta
+    # + state, write theta + state
+    total = grad_bytes + (N - 1) * P * 4 + (N - 1) * P * 4 + 2 * (1 + n_state) * P * 4
+    return dict(step=make_step(cfg.b), check=check, grad_bytes=grad_bytes, total_bytes=total,
+                launches_per_step=N + cfg.b, kernel="accumulate_arrival_kernel<%s, %s>, %d launches per step"
+                % (cfg.grad_dtype, cfg.opt["kind"], N + cfg.b), state=dict(grad=grad), extra=extra)
+
+
+def max_over_ranks(dist, values, device):
+    """Element-wise maximum of `values` over all ranks (the slowest rank sets the job's time)."""
+    if dist is None:
+        return list(values)
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_rate(world: int, bytes_per_rank_step: float, ms_per_step: float) -> float:
+    """GB/s of the whole job: every rank moves bytes_per_rank_step in the (slowest rank's) step time."""
+    return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
+
+
+def time_steps(step, steps, warmup):
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(steps):
+        step(warmup + i)
+    stop.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(stop) / steps
+
+
 def run_native(args, cfg):
     from paper_1604_00981_b200 import binding as sgdb
 
@@ -189,28 +349,14 @@ def run_native(args, cfg):
             dist.barrier()
         torch.cuda.synchronize()
 
-    W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
     seed = cfg.seed + 1000 * rank  # every rank is its own parameter-server shard
-    scales = wl.worker_scales(cfg.seed, W)
-    grad = wl.grad_matrix(seed, 0, W, P, scales, cfg.grad_dtype, dev)
-    theta = wl.theta0(seed, P, dev)
-    s0 = torch.zeros(P, device=dev)
-    s1 = torch.zeros(P, device=dev)
-    mask = torch.zeros(W, dtype=torch.uint8, device=dev)
-    order = torch.zeros(N, dtype=torch.int32, device=dev)
-    info = torch.zeros(2, dtype=torch.int32, device=dev)
-    n_sets = 16  # arrival/tag draws rotate, so the kept set differs from step to step
-    arr_d = [torch.from_numpy(wl.arrivals(cfg.seed, t, W)).to(dev) for t in range(n_sets)]
-    tag_d = [torch.from_numpy(wl.tags(cfg.seed, t, W, N) - t).to(dev) for t in range(n_sets)]  # tags relative to t = 0
-    opt = sgdb.Opt(**cfg.opt)
-    esize = grad.element_size()
-    grad_bytes = N * P * esize
-    n_state = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2}[cfg.opt["kind"]]
-    total_bytes = grad_bytes + 2 * (1 + n_state) * P * 4
-
-    def step(i):
-        opt.step = i + 1
-        sgdb.sgdb_step(grad, P, arr_d[i % n_sets], tag_d[i % n_sets], 0, N, b, theta, s0, s1, opt, mask, order, info)
+    if cfg.segments:
+        wk = setup_segmented(cfg, dev, sgdb, seed)
+    elif cfg.name.startswith("c4"):
+        wk = setup_arrivals(cfg, dev, sgdb, seed)
+    else:
+        wk = setup_flat(cfg, dev, sgdb, seed)
+    step = wk["step"]
 
     for i in range(args.warmup):
         step(i)
@@ -224,29 +370,33 @@ def run_native(args, cfg):
         stop.record()
         barrier()
     ms_total = start.elapsed_time(stop)
-    assert info.cpu().tolist()[1] == 0, "a step reported a device-side error"
-    assert bool(torch.isfinite(theta).all())
+    wk["check"]()
+    extra = wk["extra"]() if callable(wk["extra"]) else wk["extra"]
 
     # ---- end to end: gradients start in pinned host memory, new parameters are read back
-    if args.no_e2e:
-        return finish(args, cfg, dist, dev, rank, world, ms_total, None, 0, clocks, grad_bytes, total_bytes, esize)
+    flat = not cfg.segments and not cfg.name.startswith("c4")
+    if args.no_e2e or not flat or cfg.W * cfg.P * (4 if cfg.grad_dtype == "f32" else 2) > 16e9:
+        return finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, None, 0, clocks)
+    W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
+    st = wk["state"]
+    grad, theta, s0, s1, opt = st["grad"], st["theta"], st["s0"], st["s1"], st["opt"]
     e2e_steps = max(1, min(args.steps, 3))
     ws = torch.empty(sgdb.sgdb_step_host_workspace_bytes(grad.dtype, P, P, N, b), dtype=torch.uint8, device=dev)
     h_grad = torch.empty((W, P), dtype=grad.dtype, pin_memory=True)
     h_grad.copy_(grad)
-    del grad
+    del grad, st["grad"]
     h_theta = torch.empty(P, dtype=torch.float32, pin_memory=True)
     h_mask = torch.empty(W, dtype=torch.uint8, pin_memory=True)
     h_order = torch.empty(N, dtype=torch.int32, pin_memory=True)
     h_info = torch.empty(2, dtype=torch.int32, pin_memory=True)
-    h_arr = [torch.from_numpy(wl.arrivals(cfg.seed, t, W)).pin_memory() for t in range(n_sets)]
-    h_tag = [torch.from_numpy(wl.tags(cfg.seed, t, W, N) - t).pin_memory() for t in range(n_sets)]
+    h_arr = [torch.from_numpy(wl.arrivals(cfg.seed, t, W)).pin_memory() for t in range(N_SETS)]
+    h_tag = [torch.from_numpy(wl.tags(cfg.seed, t, W, N) - t).pin_memory() for t in range(N_SETS)]
 
     def host_step(i):
         opt.step = i + 1
-        st = sgdb.sgdb_step_host(h_grad, P, h_arr[i % n_sets], h_tag[i % n_sets], 0, N, b, theta, s0, s1, opt,
-                                 h_theta, h_mask, h_order, h_info, ws)
-        assert st == 0
+        status = sgdb.sgdb_step_host(h_grad, P, h_arr[i % N_SETS], h_tag[i % N_SETS], 0, N, b, theta, s0, s1, opt,
+                                     h_theta, h_mask, h_order, h_info, ws)
+        assert status == 0
 
     host_step(0)
     barrier()
@@ -257,22 +407,22 @@ def run_native(args, cfg):
     e_stop.record()
     barrier()
     e2e_ms = e_start.elapsed_time(e_stop)
-    return finish(args, cfg, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks, grad_bytes, total_bytes, esize)
+    return finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks)
 
 
-def finish(args, cfg, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks, grad_bytes, total_bytes, esize):
-    W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
-    # ---- max over ranks
-    if dist is not None:
-        tt = torch.tensor([ms_total, e2e_ms or 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total, e2e_ms = float(tt[0]), (float(tt[1]) if e2e_ms is not None else None)
+def finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks):
+    W, N, b = cfg.W, cfg.N, cfg.b
+    P = wk.get("P", cfg.P)
+    grad_bytes, total_bytes = wk["grad_bytes"], wk["total_bytes"]
+    esize = 4 if cfg.grad_dtype == "f32" else 2
+    ms_total, e2e_max = max_over_ranks(dist, [ms_total, e2e_ms or 0.0], dev)
+    e2e_ms = e2e_max if e2e_ms is not None else None
     ms_per_step = ms_total / args.steps
-    value = world * grad_bytes / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_rate(world, grad_bytes, ms_per_step)
     total_gbs_per_gpu = total_bytes / (ms_per_step * 1e-3) / 1e9
     e2e = None
     if e2e_ms is not None:
-        e2e = {"value": world * grad_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": UNIT,
+        e2e = {"value": whole_job_rate(world, grad_bytes, e2e_ms / e2e_steps), "unit": UNIT,
                "h2d_bytes_per_step": N * P * esize + W * 8, "d2h_bytes_per_step": P * 4 + W + N * 4 + 16,
                "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps}
 
@@ -280,10 +430,11 @@ def finish(args, cfg, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clock
         peak, peak_kind = measured_hbm_peak()
         digest = kernel_source_digest()
         traffic = None
-        if NCU_TRAFFIC["src_digest"] == digest and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] is not None:
+        if (cfg.name == "c1_inception_rmsprop" and NCU_TRAFFIC["src_digest"] == digest
+                and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] is not None):
             traffic = NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] * total_bytes
         cpu = None
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and cfg.name.startswith("c1"):
             P_sample = P // 4
             sec, gbs = oracle_sample_run(cfg, P_sample, steps=10, warmup=1)
             cpu = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
@@ -295,20 +446,21 @@ def finish(args, cfg, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clock
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": cfg.name, "P": P, "W": W, "N": N, "b": b, "optimizer": cfg.opt["kind"],
                        "grad_dtype": cfg.grad_dtype, "sharding": "one parameter-server column shard of P per GPU",
-                       "l2": "inputs larger than L2: %.2f GB of gradient rows and %.0f MB of parameters and state per step"
-                             % (grad_bytes / 1e9, (total_bytes - grad_bytes) / 2e6)},
+                       "l2": "inputs larger than L2 (126 MB): %.3f GB of gradient rows and %.1f MB of parameters and "
+                             "state per step" % (grad_bytes / 1e9, (total_bytes - grad_bytes) / 2e6)},
             "step_us": ms_per_step * 1e3,
             "total_gbs_per_gpu": total_gbs_per_gpu,
             "pct_of_nominal_8tbs": 100.0 * total_gbs_per_gpu / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": total_gbs_per_gpu, "peak": peak, "unit": "GB/s",
                          "frac": total_gbs_per_gpu / peak, "traffic": traffic, "peak_source": peak_kind,
-                         "kernel": "stream_rows_kernel<float, rmsprop> (the step is this one launch)",
-                         "algorithmic_bytes_per_launch": total_bytes},
+                         "kernel": wk["kernel"], "algorithmic_bytes_per_step": total_bytes},
             "e2e": e2e,
-            "gpu_launches": args.steps,  # one fused launch per step (selection is the kernel's prologue)
+            "gpu_launches": wk["launches_per_step"] * args.steps,
             "clocks": clocks.summary(),
             "cpu_baseline": cpu,
         }
+        if extra:
+            line["extra"] = extra
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -322,12 +474,14 @@ def main():
     ap.add_argument("--impl", choices=["native", "reference"], default="native")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--workload", choices=["c0", "c1", "c2", "c3", "c4"], default="c1",
+                    help="c1 (default) is the benchmark workload; the others time the remaining seeded workloads")
     ap.add_argument("--columns", type=int, default=0,
                     help="override P with a smaller column count (profiler captures); not the benchmark workload")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "native":
         args.warmup = 3
-    cfg = wl.CONFIGS[1]
+    cfg = wl.CONFIGS[{"c0": 0, "c1": 1, "c2": 2, "c3": 3, "c4": 4}[args.workload]]
     if args.columns > 0:
         import dataclasses
 

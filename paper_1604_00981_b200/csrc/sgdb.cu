@@ -26,10 +26,19 @@ constexpr int kMaxDevices = 64;
 #ifndef SGDB_CH
 #define SGDB_CH 2
 #endif
+#ifndef SGDB_CH_BF16
+#define SGDB_CH_BF16 SGDB_CH
+#endif
 constexpr int kNT = SGDB_NT;
-constexpr int kCH = SGDB_CH;
-constexpr int kStageBytes = kNT * kCH * 16;
-constexpr int kDefaultStages = 6;
+template <typename GT>
+struct Shape {  // 16-byte chunks per thread and row, per gradient type
+  static constexpr int kCH = SGDB_CH;
+};
+template <>
+struct Shape<BF16> {
+  static constexpr int kCH = SGDB_CH_BF16;
+};
+constexpr int kDefaultStages = 7;
 constexpr int kDefaultCtasPerSm = 2;
 
 struct DeviceInfo {
@@ -40,6 +49,7 @@ struct DeviceInfo {
 DeviceInfo g_dev[kMaxDevices];
 int g_stages = kDefaultStages;
 int g_ctas_per_sm = kDefaultCtasPerSm;
+int g_arrival_blocks_per_sm = 4;
 
 bool is_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -136,6 +146,8 @@ sgdb_status_t launch_stream_t(const StreamParams& p_in, long long total_tiles_hi
   sgdb_status_t st = device_info(&dev);
   if (st != SGDB_OK) return st;
   StreamParams p = p_in;
+  constexpr int kCH = Shape<GT>::kCH;
+  constexpr int kStageBytes = kNT * kCH * 16;
   auto kernel = stream_rows_kernel<GT, EP, kNT, kCH>;
 
   // shared memory: ring + 2 barriers per slot + order[N] + tile prefix[S + 1]
@@ -184,7 +196,8 @@ sgdb_status_t launch_stream(int dt, int ep, const StreamParams& p, long long til
 }
 
 long long tiles_of(int dt, long long len) {
-  const long long tile = static_cast<long long>(kNT) * kCH * (dt == SGDB_BF16 ? 8 : 4);
+  const long long tile = dt == SGDB_BF16 ? static_cast<long long>(kNT) * Shape<BF16>::kCH * 8
+                                         : static_cast<long long>(kNT) * Shape<float>::kCH * 4;
   return (len + tile - 1) / tile;
 }
 
@@ -356,8 +369,8 @@ sgdb_status_t sgdb_accumulate_arrival(const void* d_row, sgdb_dtype_t dt, int32_
   ArrivalParams p{d_row, row_tag, t, N, P, d_acc, d_counter, d_theta, d_state0, d_state1, d_info, h};
   const int V = dt == SGDB_BF16 ? 8 : 4;
   const long long chunks = (P + V - 1) / V;
-  long long grid = (chunks + 255) / 256;
-  const long long cap = static_cast<long long>(dev->sms) * 8;
+  long long grid = (chunks + 4 * 256 - 1) / (4 * 256);  // 4 chunks per thread and pass
+  const long long cap = static_cast<long long>(dev->sms) * g_arrival_blocks_per_sm;
   if (grid > cap) grid = cap;
   if (row_tag != t || grid < 1) grid = 1;  // a wrongly tagged gradient only updates the bookkeeping
   cudaStream_t s = static_cast<cudaStream_t>(stream);

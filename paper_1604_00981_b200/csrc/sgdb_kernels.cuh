@@ -286,56 +286,107 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
     for (int tile = blockIdx.x; tile < total_tiles && !timed_out; tile += gridDim.x) {
       const TileDesc<GT> td = locate_tile<GT, TILE>(p, prefix_s, tile);
 
-      // theta and state of this tile are requested now and used after the row loop
-      float th[CH][V], s0[CH][V], s1[CH][V];
-#pragma unroll
-      for (int c = 0; c < CH; ++c) {
-        const int o = (tid + c * NT) * V;
-        const int n = td.ncols - o;
-        if (n > 0) {
-          const bool vec = td.vec_ok && n >= V;
-          if (Rule::kTheta) load_floats<V>(td.theta + o, vec, n, th[c]);
-          if (Rule::kState0) load_floats<V>(td.s0 + o, vec, n, s0[c]);
-          if (Rule::kState1) load_floats<V>(td.s1 + o, vec, n, s1[c]);
-        }
-      }
-
       float acc[CH][V];
 #pragma unroll
       for (int c = 0; c < CH; ++c)
 #pragma unroll
         for (int e = 0; e < V; ++e) acc[c][e] = 0.0f;
 
-      for (int k = 0; k < N; ++k) {
+      // columns of this thread that the bulk copy did not deliver (ragged end, unaligned
+      // segment) are read straight from global memory, row by row, in the same order
+      auto add_row_tail = [&](int k) {
         const GT* row = td.grad + static_cast<long long>(order_s[k]) * td.ld;
-        const unsigned char* stage = smem + static_cast<size_t>(s) * STAGE_BYTES;
-        if (td.bulk_cols > 0) {
-          if (!mbar_wait(full_addr + 8u * s, phase, &s_abort)) {
-            timed_out = true;
-            break;
-          }
-        }
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
           const int o = (tid + c * NT) * V;
-          if (o + V <= td.bulk_cols) {
-            const uint4 v = *reinterpret_cast<const uint4*>(stage + static_cast<size_t>(o) * sizeof(GT));
-            float x[V];
-            Tr::unpack(v, x);
-#pragma unroll
-            for (int e = 0; e < V; ++e) acc[c][e] = __fadd_rn(acc[c][e], x[e]);
-          } else if (o < td.ncols) {
+          if (o + V > td.bulk_cols && o < td.ncols) {
 #pragma unroll
             for (int e = 0; e < V; ++e)
               if (o + e < td.ncols) acc[c][e] = __fadd_rn(acc[c][e], Tr::widen(row[o + e]));
           }
         }
-        if (td.bulk_cols > 0) {
-          __syncwarp();
-          if (lane == 0) mbar_arrive(empty_addr + 8u * s);
+      };
+      const bool has_tail = td.bulk_cols < td.ncols;
+
+      if (td.bulk_cols == 0) {
+        for (int k = 0; k < N; ++k) add_row_tail(k);
+      } else {
+        int k = 0;
+        // two rows per pass: both slots are waited for and read before the dependent adds
+        for (; k + 1 < N; k += 2) {
+          const int sa = s;
+          const uint32_t pa = phase;
           if (++s == stages) {
             s = 0;
             phase ^= 1u;
+          }
+          const int sb = s;
+          const uint32_t pb = phase;
+          if (++s == stages) {
+            s = 0;
+            phase ^= 1u;
+          }
+          if (!mbar_wait(full_addr + 8u * sa, pa, &s_abort) || !mbar_wait(full_addr + 8u * sb, pb, &s_abort)) {
+            timed_out = true;
+            break;
+          }
+          const unsigned char* stage_a = smem + static_cast<size_t>(sa) * STAGE_BYTES;
+          const unsigned char* stage_b = smem + static_cast<size_t>(sb) * STAGE_BYTES;
+          uint4 va[CH], vb[CH];
+#pragma unroll
+          for (int c = 0; c < CH; ++c) {
+            const int o = (tid + c * NT) * V;
+            if (o + V <= td.bulk_cols) {
+              va[c] = *reinterpret_cast<const uint4*>(stage_a + static_cast<size_t>(o) * sizeof(GT));
+              vb[c] = *reinterpret_cast<const uint4*>(stage_b + static_cast<size_t>(o) * sizeof(GT));
+            }
+          }
+#pragma unroll
+          for (int c = 0; c < CH; ++c) {
+            const int o = (tid + c * NT) * V;
+            if (o + V <= td.bulk_cols) {
+              float x[V];
+              Tr::unpack(va[c], x);
+#pragma unroll
+              for (int e = 0; e < V; ++e) acc[c][e] = __fadd_rn(acc[c][e], x[e]);
+              Tr::unpack(vb[c], x);
+#pragma unroll
+              for (int e = 0; e < V; ++e) acc[c][e] = __fadd_rn(acc[c][e], x[e]);
+            }
+          }
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(empty_addr + 8u * sa);
+            mbar_arrive(empty_addr + 8u * sb);
+          }
+          if (has_tail) {
+            add_row_tail(k);
+            add_row_tail(k + 1);
+          }
+        }
+        if (!timed_out && k < N) {  // N odd: the last row on its own
+          if (!mbar_wait(full_addr + 8u * s, phase, &s_abort)) {
+            timed_out = true;
+          } else {
+            const unsigned char* stage = smem + static_cast<size_t>(s) * STAGE_BYTES;
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+              const int o = (tid + c * NT) * V;
+              if (o + V <= td.bulk_cols) {
+                const uint4 v = *reinterpret_cast<const uint4*>(stage + static_cast<size_t>(o) * sizeof(GT));
+                float x[V];
+                Tr::unpack(v, x);
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[c][e] = __fadd_rn(acc[c][e], x[e]);
+              }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_addr + 8u * s);
+            if (++s == stages) {
+              s = 0;
+              phase ^= 1u;
+            }
+            if (has_tail) add_row_tail(k);
           }
         }
       }
@@ -353,11 +404,19 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
           if (EP == EP_MEAN) {
             store_floats<V>(td.theta + o, vec, n, g);
           } else {
+            // theta and state are loaded here, not ahead of the row loop: holding them in
+            // registers through the loop measured no faster for fp32 rows and slower for bf16
+            // rows (spills at two resident blocks); the other block on the SM and the ring,
+            // which keeps filling, cover this latency
+            float th[V], s0[V], s1[V];
+            if (Rule::kTheta) load_floats<V>(td.theta + o, vec, n, th);
+            if (Rule::kState0) load_floats<V>(td.s0 + o, vec, n, s0);
+            if (Rule::kState1) load_floats<V>(td.s1 + o, vec, n, s1);
 #pragma unroll
-            for (int e = 0; e < V; ++e) apply_rule<EP>(p.h, g[e], th[c][e], s0[c][e], s1[c][e]);
-            store_floats<V>(td.theta + o, vec, n, th[c]);
-            if (Rule::kState0) store_floats<V>(td.s0 + o, vec, n, s0[c]);
-            if (Rule::kState1) store_floats<V>(td.s1 + o, vec, n, s1[c]);
+            for (int e = 0; e < V; ++e) apply_rule<EP>(p.h, g[e], th[e], s0[e], s1[e]);
+            store_floats<V>(td.theta + o, vec, n, th);
+            if (Rule::kState0) store_floats<V>(td.s0 + o, vec, n, s0);
+            if (Rule::kState1) store_floats<V>(td.s1 + o, vec, n, s1);
           }
         }
       }
@@ -424,7 +483,7 @@ struct ArrivalParams {
 };
 
 template <typename GT, int EP>
-__global__ void __launch_bounds__(256) accumulate_arrival_kernel(const ArrivalParams p) {
+__global__ void __launch_bounds__(256, 4) accumulate_arrival_kernel(const ArrivalParams p) {
   using Tr = GradTraits<GT>;
   using Rule = RuleTraits<EP>;
   constexpr int V = Tr::kVec;
@@ -445,37 +504,74 @@ __global__ void __launch_bounds__(256) accumulate_arrival_kernel(const ArrivalPa
     const float n_as_float = static_cast<float>(p.N);
     const long long chunks = (p.P + V - 1) / V;
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-    for (long long q = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; q < chunks; q += stride) {
-      const long long i = q * V;
-      const long long rest = p.P - i;
-      const int n = rest < V ? static_cast<int>(rest) : V;
-      const bool vec = n == V;
-      float x[V], a[V];
-      if (vec && row_vec) {
-        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(row + i));
-        Tr::unpack(v, x);
-      } else {
+    const long long first_chunk = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (!last) {
+      // U chunks per thread and pass, all loads issued before the first use: enough bytes
+      // in flight per SM for a stream that reads two arrays and writes one.
+      constexpr int U = 16 / V;  // 64 bytes of the row per thread and pass
+      for (long long q0 = first_chunk; q0 < chunks; q0 += stride * U) {
+        float x[U][V], a[U][V];
+        int n[U];
 #pragma unroll
-        for (int e = 0; e < V; ++e) x[e] = e < n ? Tr::widen(row[i + e]) : 0.0f;
+        for (int u = 0; u < U; ++u) {
+          const long long q = q0 + u * stride;
+          const long long i = q * V;
+          const long long rest = p.P - i;
+          n[u] = q < chunks ? (rest < V ? static_cast<int>(rest) : V) : 0;
+          if (n[u] > 0) {
+            if (n[u] == V && row_vec) {
+              const uint4 v = __ldcs(reinterpret_cast<const uint4*>(row + i));
+              Tr::unpack(v, x[u]);
+            } else {
+#pragma unroll
+              for (int e = 0; e < V; ++e) x[u][e] = e < n[u] ? Tr::widen(row[i + e]) : 0.0f;
+            }
+            if (first) {
+#pragma unroll
+              for (int e = 0; e < V; ++e) a[u][e] = 0.0f;
+            } else {
+              load_floats<V>(p.acc + i, n[u] == V, n[u], a[u]);
+            }
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          if (n[u] > 0) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) a[u][e] = __fadd_rn(a[u][e], x[u][e]);
+            store_floats<V>(p.acc + (q0 + u * stride) * V, n[u] == V, n[u], a[u]);
+          }
+        }
       }
-      if (first) {
+    } else {
+      // the gradient that completes the set: mean and optimizer rule in the same pass
+      for (long long q = first_chunk; q < chunks; q += stride) {
+        const long long i = q * V;
+        const long long rest = p.P - i;
+        const int n = rest < V ? static_cast<int>(rest) : V;
+        const bool vec = n == V;
+        float x[V], a[V], th[V], s0[V], s1[V];
+        if (vec && row_vec) {
+          const uint4 v = __ldcs(reinterpret_cast<const uint4*>(row + i));
+          Tr::unpack(v, x);
+        } else {
 #pragma unroll
-        for (int e = 0; e < V; ++e) a[e] = 0.0f;
-      } else {
-        load_floats<V>(p.acc + i, vec, n, a);
-      }
+          for (int e = 0; e < V; ++e) x[e] = e < n ? Tr::widen(row[i + e]) : 0.0f;
+        }
+        if (first) {
 #pragma unroll
-      for (int e = 0; e < V; ++e) a[e] = __fadd_rn(a[e], x[e]);
-      if (!last) {
-        store_floats<V>(p.acc + i, vec, n, a);
-      } else {
-        float th[V], s0[V], s1[V];
+          for (int e = 0; e < V; ++e) a[e] = 0.0f;
+        } else {
+          load_floats<V>(p.acc + i, vec, n, a);
+        }
         load_floats<V>(p.theta + i, vec, n, th);
         if (Rule::kState0) load_floats<V>(p.s0 + i, vec, n, s0);
         if (Rule::kState1) load_floats<V>(p.s1 + i, vec, n, s1);
 #pragma unroll
-        for (int e = 0; e < V; ++e)
+        for (int e = 0; e < V; ++e) {
+          a[e] = __fadd_rn(a[e], x[e]);
           apply_rule<EP>(p.h, __fdiv_rn(a[e], n_as_float), th[e], s0[e], s1[e]);
+        }
         store_floats<V>(p.theta + i, vec, n, th);
         if (Rule::kState0) store_floats<V>(p.s0 + i, vec, n, s0);
         if (Rule::kState1) store_floats<V>(p.s1 + i, vec, n, s1);
