@@ -1,0 +1,88 @@
+"""Do the pins bite?  Plausible mistakes are planted in copies of the oracle's C source (on the CPU,
+never in the GPU path); every mutant must make at least one pin of test_oracle_pins.py fail."""
+import ctypes
+import os
+import subprocess
+
+import pytest
+
+import oracle
+import test_oracle_pins as pins
+
+SRC = os.path.join(os.path.dirname(oracle.__file__), "sgdb_oracle.c")
+
+# (name, text in the source, replacement)
+MUTANTS = [
+    ("divide_by_all_workers", "mean[i] = sum / (double)N;", "mean[i] = sum / (double)(N + 0 * ld + 1);"),
+    ("stale_gradients_kept", "if (tags[w] != t) continue;", "if (tags[w] > t) continue;"),
+    ("future_gradients_kept", "if (tags[w] != t) continue;", "if (tags[w] < t) continue;"),
+    ("infinite_arrivals_kept", "if (!isfinite(arrival[w])) continue;", "if (isnan(arrival[w])) continue;"),
+    ("ties_by_higher_id", "return a < b;", "return a > b;"),
+    ("latest_first", "if (arrival[a] < arrival[b]) return 1;\n  if (arrival[a] > arrival[b]) return 0;",
+     "if (arrival[a] > arrival[b]) return 1;\n  if (arrival[a] < arrival[b]) return 0;"),
+    ("keeps_one_too_few", "for (int32_t k = 0; k < N; ++k) { /* the server stops waiting at |G| = N */",
+     "for (int32_t k = 0; k + 1 < N; ++k) {"),
+    ("row_major_transposed", "(int64_t)order[k] * ld + i", "(int64_t)i * N + order[k]"),
+    ("sums_first_n_rows", "grad_at(grad, dtype, (int64_t)order[k] * ld + i)", "grad_at(grad, dtype, (int64_t)k * ld + i)"),
+    ("bf16_low_half", "((uint32_t)bits) << 16", "((uint32_t)bits)"),
+    ("sgd_sign", "theta[i] = theta[i] - opt->lr * g;", "theta[i] = theta[i] + opt->lr * g;"),
+    ("momentum_scaled_gradient", "s0[i] = opt->momentum * s0[i] + g;", "s0[i] = opt->momentum * s0[i] + (1.0 - opt->momentum) * g;"),
+    ("rmsprop_eps_outside", "sqrt(s0[i] + opt->eps)", "(sqrt(s0[i]) + opt->eps)"),
+    ("rmsprop_no_decay_complement", "(1.0 - opt->decay) * g * g", "g * g"),
+    ("rmsprop_lr_outside_momentum", "s1[i] = opt->momentum * s1[i] + opt->lr * g / sqrt(s0[i] + opt->eps);\n        theta[i] = theta[i] - s1[i];",
+     "s1[i] = opt->momentum * s1[i] + g / sqrt(s0[i] + opt->eps);\n        theta[i] = theta[i] - opt->lr * s1[i];"),
+    ("adam_no_bias_correction", "double m_hat = s0[i] / (1.0 - pow(opt->beta1, (double)opt->step));", "double m_hat = s0[i];"),
+    ("adam_eps_inside", "(sqrt(v_hat) + opt->eps)", "sqrt(v_hat + opt->eps)"),
+    ("adam_moments_swapped", "s1[i] = opt->beta2 * s1[i] + (1.0 - opt->beta2) * g * g;", "s1[i] = opt->beta1 * s1[i] + (1.0 - opt->beta1) * g * g;"),
+    ("arrival_counts_stale", "if (row_tag != t || t < state[2] || state[0] >= N) {", "if (t < state[2] || state[0] >= N) {"),
+    ("arrival_never_closes", "state[2] = t + 1;", "state[2] = state[2];"),
+    ("arrival_divides_late", "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)N;", "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)(N + 1);"),
+    ("arrival_keeps_old_sum", "if (state[0] == 0)\n    for (int64_t i = 0; i < P; ++i) acc[i] = 0.0; /* G = {} */", ""),
+]
+
+PIN_TESTS = [getattr(pins, n) for n in dir(pins) if n.startswith("test_")]
+
+
+def _run_pin(fn):
+    marks = [m for m in getattr(fn, "pytestmark", []) if m.name == "parametrize"]
+    if not marks:
+        fn()
+        return
+    names = [n.strip() for n in marks[0].args[0].split(",")]
+    for values in marks[0].args[1]:
+        values = values if isinstance(values, (tuple, list)) else (values,)
+        fn(**dict(zip(names, values)))
+
+
+@pytest.mark.parametrize("name,old,new", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_mutant_is_caught_by_a_pin(tmp_path, name, old, new):
+    text = open(SRC).read()
+    assert text.count(old) >= 1, "mutation site not found: the oracle changed, update this list"
+    mutated = text.replace(old, new, 1)
+    c_path, so_path = tmp_path / "mutant.c", tmp_path / "mutant.so"
+    c_path.write_text(mutated)
+    subprocess.run(["gcc", "-O1", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off", "-o", str(so_path), str(c_path), "-lm"],
+                   check=True)
+    lib = ctypes.CDLL(str(so_path))
+    for fn_name in ("oracle_select", "oracle_aggregate", "oracle_update", "oracle_step", "oracle_accumulate_arrival"):
+        getattr(lib, fn_name).restype = ctypes.c_int
+    oracle._load()
+    saved = oracle._lib
+    oracle._lib = lib
+    caught = []
+    try:
+        for fn in PIN_TESTS:
+            try:
+                _run_pin(fn)
+            except AssertionError:
+                caught.append(fn.__name__)
+            except Exception as e:  # a crash of the mutant inside a pin also exposes it
+                caught.append(fn.__name__ + ":" + type(e).__name__)
+    finally:
+        oracle._lib = saved
+    assert caught, "no pin noticed the planted mistake '%s'" % name
+
+
+def test_unmutated_oracle_passes_every_pin_through_the_same_driver():
+    for fn in PIN_TESTS:
+        _run_pin(fn)

@@ -341,6 +341,17 @@ def test_rmsprop_eps_is_inside_the_root_and_state_is_callers():
     assert th[0] == -m[0]
 
 
+def test_rmsprop_learning_rate_enters_the_momentum_buffer():
+    """With decay 0 and eps 0 the scaled gradient is sign(g); lr 1 then lr 4, momentum 0.5:
+    m_1 = 1, m_2 = 0.5 * 1 + 4 = 4.5, theta_2 = theta_0 - 5.5 (lr applied outside the buffer would give -7)."""
+    g = np.array([3.0, -2.0])
+    th, s, m = np.array([10.0, 10.0]), np.zeros(2), np.zeros(2)
+    oracle.update(th, s, m, g, oracle.Opt(kind=oracle.RMSPROP, lr=1.0, decay=0.0, momentum=0.5, eps=0.0))
+    assert th.tolist() == [9.0, 11.0] and m.tolist() == [1.0, -1.0]
+    oracle.update(th, s, m, g, oracle.Opt(kind=oracle.RMSPROP, lr=4.0, decay=0.0, momentum=0.5, eps=0.0))
+    assert m.tolist() == [4.5, -4.5] and th.tolist() == [4.5, 15.5]
+
+
 def test_adam_closed_form_every_step():
     lr, eps, k = 1e-3, 1e-8, 9
     traj = _run_constant(oracle.ADAM, G_CONST, k, lr=lr, beta1=0.9, beta2=0.999, eps=eps)
