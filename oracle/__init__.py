@@ -83,8 +83,11 @@ def _load():
             "oracle_update",
             "oracle_step",
             "oracle_accumulate_arrival",
+            "oracle_step_ema",
         ):
             getattr(lib, name).restype = ctypes.c_int
+        lib.oracle_ema.restype = None
+        lib.oracle_learning_rate.restype = ctypes.c_double
         _lib = lib
     return _lib
 
@@ -161,6 +164,41 @@ def step(grad, P: int, arrival, tags, t: int, N: int, b: int, theta, s0, s1, opt
         ctypes.byref(c), _p(mask), _p(order), ctypes.byref(n_valid),
     )
     return rc, mask, order, n_valid.value
+
+
+def ema(avg, theta, alpha: float) -> None:
+    """avg <- alpha * avg + (1 - alpha) * theta, in place on the fp64 array avg (Section 1.1)."""
+    assert avg.dtype == np.float64 and avg.flags.c_contiguous
+    theta = np.ascontiguousarray(theta, dtype=np.float64)
+    _load().oracle_ema(_p(avg), _p(theta), ctypes.c_int64(len(avg)), ctypes.c_double(alpha))
+
+
+def step_ema(grad, P: int, arrival, tags, t: int, N: int, b: int, theta, s0, s1, opt: Opt, avg, alpha: float,
+             ld: int | None = None):
+    """One iteration of Algorithm 4 with its last line (the average of the pre-update parameters)."""
+    W = N + b
+    g, dt = _grad(grad)
+    ld = g.shape[1] if ld is None else ld
+    arrival = np.ascontiguousarray(arrival, dtype=np.float32)
+    tags = np.ascontiguousarray(tags, dtype=np.int32)
+    for a in (theta, s0, s1, avg):
+        assert a is None or (a.dtype == np.float64 and a.flags.c_contiguous)
+    mask = np.zeros(W, dtype=np.uint8)
+    order = np.full(N, -1, dtype=np.int32)
+    n_valid = ctypes.c_int32(0)
+    c = opt._c()
+    rc = _load().oracle_step_ema(
+        _p(g), ctypes.c_int(dt), ctypes.c_int64(P), ctypes.c_int64(ld), _p(arrival), _p(tags),
+        ctypes.c_int32(t), ctypes.c_int32(N), ctypes.c_int32(b), _p(theta), _p(s0), _p(s1),
+        ctypes.byref(c), _p(avg), ctypes.c_double(alpha), _p(mask), _p(order), ctypes.byref(n_valid),
+    )
+    return rc, mask, order, n_valid.value
+
+
+def learning_rate(gamma0: float, beta: float, t: int, N: int, T: float) -> float:
+    """gamma0 * beta^(t N / (2 T)) (Appendix A.2, A.3)."""
+    return float(_load().oracle_learning_rate(ctypes.c_double(gamma0), ctypes.c_double(beta), ctypes.c_int64(t),
+                                              ctypes.c_int64(N), ctypes.c_double(T)))
 
 
 def new_server_state():

@@ -172,6 +172,40 @@ int oracle_step(const void *grad, int dtype, int64_t P, int64_t ld, const float 
 }
 
 /*
+ * Section 1.1 / the last line of Algorithm 4: the exponential moving average of the
+ * parameters, avg(t) = alpha * avg(t-1) + (1 - alpha) * theta(t).  The paper does not
+ * define avg(-1); the caller initialises it (the tests use theta(0)).
+ */
+void oracle_ema(double *avg, const double *theta, int64_t P, double alpha) {
+  for (int64_t i = 0; i < P; ++i) avg[i] = alpha * avg[i] + (1.0 - alpha) * theta[i];
+}
+
+/*
+ * One iteration of Algorithm 4 including its last line.  As printed, iteration t
+ * computes theta(t+1) from theta(t) and then averages theta(t): the average sees
+ * the parameters as they were before this iteration's update.
+ */
+int oracle_step_ema(const void *grad, int dtype, int64_t P, int64_t ld, const float *arrival,
+                    const int32_t *tags, int32_t t, int32_t N, int32_t b, double *theta, double *s0,
+                    double *s1, const oracle_opt_t *opt, double *avg, double alpha, uint8_t *mask,
+                    int32_t *order, int32_t *n_valid) {
+  double *theta_t = (double *)malloc(sizeof(double) * (size_t)(P > 0 ? P : 1));
+  memcpy(theta_t, theta, sizeof(double) * (size_t)P);
+  int rc = oracle_step(grad, dtype, P, ld, arrival, tags, t, N, b, theta, s0, s1, opt, mask, order, n_valid);
+  if (rc == ORACLE_OK) oracle_ema(avg, theta_t, P, alpha);
+  free(theta_t);
+  return rc;
+}
+
+/*
+ * Appendix A.2 / A.3: learning rate after t iterations, gamma0 * beta^(t N / (2 T)) with
+ * T = |X| / B mini-batches in the data set; N = 1 is the asynchronous schedule.
+ */
+double oracle_learning_rate(double gamma0, double beta, int64_t t, int64_t N, double T) {
+  return gamma0 * pow(beta, (double)t * (double)N / (2.0 * T));
+}
+
+/*
  * Algorithm 4's while loop, one received gradient per call.
  *   state[0] = |G| so far, state[1] = gradients received so far,
  *   state[2] = lowest iteration still open (the server's own t).

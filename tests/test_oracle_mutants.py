@@ -34,6 +34,11 @@ MUTANTS = [
     ("adam_no_bias_correction", "double m_hat = s0[i] / (1.0 - pow(opt->beta1, (double)opt->step));", "double m_hat = s0[i];"),
     ("adam_eps_inside", "(sqrt(v_hat) + opt->eps)", "sqrt(v_hat + opt->eps)"),
     ("adam_moments_swapped", "s1[i] = opt->beta2 * s1[i] + (1.0 - opt->beta2) * g * g;", "s1[i] = opt->beta1 * s1[i] + (1.0 - opt->beta1) * g * g;"),
+    ("ema_weights_swapped", "avg[i] = alpha * avg[i] + (1.0 - alpha) * theta[i];", "avg[i] = (1.0 - alpha) * avg[i] + alpha * theta[i];"),
+    ("ema_of_updated_parameters", "if (rc == ORACLE_OK) oracle_ema(avg, theta_t, P, alpha);", "if (rc == ORACLE_OK) oracle_ema(avg, theta, P, alpha);"),
+    ("ema_moves_without_update", "if (rc == ORACLE_OK) oracle_ema(avg, theta_t, P, alpha);", "oracle_ema(avg, theta_t, P, alpha);"),
+    ("schedule_without_the_half", "(double)t * (double)N / (2.0 * T)", "(double)t * (double)N / T"),
+    ("schedule_ignores_workers", "(double)t * (double)N / (2.0 * T)", "(double)t / (2.0 * T)"),
     ("arrival_counts_stale", "if (row_tag != t || t < state[2] || state[0] >= N) {", "if (t < state[2] || state[0] >= N) {"),
     ("arrival_never_closes", "state[2] = t + 1;", "state[2] = state[2];"),
     ("arrival_divides_late", "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)N;", "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)(N + 1);"),
@@ -64,8 +69,11 @@ def test_mutant_is_caught_by_a_pin(tmp_path, name, old, new):
     subprocess.run(["gcc", "-O1", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off", "-o", str(so_path), str(c_path), "-lm"],
                    check=True)
     lib = ctypes.CDLL(str(so_path))
-    for fn_name in ("oracle_select", "oracle_aggregate", "oracle_update", "oracle_step", "oracle_accumulate_arrival"):
+    for fn_name in ("oracle_select", "oracle_aggregate", "oracle_update", "oracle_step", "oracle_accumulate_arrival",
+                    "oracle_step_ema"):
         getattr(lib, fn_name).restype = ctypes.c_int
+    lib.oracle_ema.restype = None
+    lib.oracle_learning_rate.restype = ctypes.c_double
     oracle._load()
     saved = oracle._lib
     oracle._lib = lib

@@ -407,3 +407,52 @@ def test_accumulate_on_arrival_equals_batched(kind, dtype):
         np.testing.assert_allclose(s0_a, s0_b, rtol=1e-13, atol=1e-14)
         np.testing.assert_allclose(s1_a, s1_b, rtol=1e-13, atol=1e-14)
         leftovers = [(grad[w], int(tags[w])) for w in range(W) if mask[w] == 0 and tags[w] == t][:1]
+
+
+# ---------------------------------------------------------------- parameter average and learning-rate schedule
+
+
+def test_ema_closed_form_under_sgd_with_constant_gradient():
+    """theta(t) = theta0 - c t with c = lr g.  With avg(-1) = theta0 the recurrence
+    avg(t) = alpha avg(t-1) + (1 - alpha) theta(t) solves to theta0 - c (t - alpha (1 - alpha^t) / (1 - alpha))."""
+    W, N, P, lr, alpha = 4, 4, 3, 0.5, 0.75
+    g = np.array([2.0, -1.0, 0.25])
+    grad = np.repeat(g[None, :], W, axis=0).astype(np.float32)
+    arrival, tags = np.arange(W, dtype=np.float32), None
+    theta0 = np.array([1.0, 2.0, 3.0])
+    theta, avg = theta0.copy(), theta0.copy()
+    for t in range(12):
+        tags = np.full(W, t, np.int32)
+        rc, *_ = oracle.step_ema(grad, P, arrival, tags, t, N, 0, theta, None, None,
+                                 oracle.Opt(kind=oracle.SGD, lr=lr), avg, alpha)
+        assert rc == oracle.OK
+        d = t - alpha * (1 - alpha ** t) / (1 - alpha)
+        np.testing.assert_allclose(avg, theta0 - lr * g * d, rtol=1e-13, atol=1e-14)
+        np.testing.assert_allclose(theta, theta0 - lr * g * (t + 1), rtol=1e-13)
+
+
+def test_ema_sees_the_parameters_before_the_update_and_limits_of_alpha():
+    grad = np.ones((2, 2), np.float32)
+    arrival, tags = np.array([1, 2], np.float32), np.zeros(2, np.int32)
+    opt = oracle.Opt(kind=oracle.SGD, lr=1.0)
+    theta, avg = np.array([5.0, 7.0]), np.array([100.0, 100.0])
+    oracle.step_ema(grad, 2, arrival, tags, 0, 2, 0, theta, None, None, opt, avg, 0.0)
+    assert avg.tolist() == [5.0, 7.0] and theta.tolist() == [4.0, 6.0]  # alpha = 0: avg = theta(t), not theta(t+1)
+    oracle.step_ema(grad, 2, arrival, tags, 0, 2, 0, theta, None, None, opt, avg, 1.0)
+    assert avg.tolist() == [5.0, 7.0] and theta.tolist() == [3.0, 5.0]  # alpha = 1: avg frozen
+    avg2 = np.array([8.0, 0.0])
+    oracle.ema(avg2, np.array([0.0, 8.0]), 0.25)
+    assert avg2.tolist() == [2.0, 6.0]
+    # too few current gradients: nothing moves, the average included
+    rc, *_ = oracle.step_ema(grad, 2, arrival, np.array([0, 9], np.int32), 0, 2, 0, theta, None, None, opt, avg, 0.0)
+    assert rc == oracle.INSUFFICIENT and avg.tolist() == [5.0, 7.0] and theta.tolist() == [3.0, 5.0]
+
+
+def test_learning_rate_schedule():
+    """Appendix A: gamma0 * 0.94^(t N / (2 T)): one factor of beta every two passes over the data."""
+    T = 40_000.0  # mini-batches per pass
+    assert oracle.learning_rate(4.5, 0.94, 0, 100, T) == 4.5
+    assert oracle.learning_rate(4.5, 0.94, 800, 100, T) == pytest.approx(4.5 * 0.94, rel=1e-14)  # t N = 2 T
+    assert oracle.learning_rate(4.5, 0.94, 1600, 100, T) == pytest.approx(4.5 * 0.94 ** 2, rel=1e-14)
+    assert oracle.learning_rate(0.045, 0.94, 80_000, 1, T) == pytest.approx(0.045 * 0.94, rel=1e-14)  # asynchronous rule
+    assert oracle.learning_rate(1.0, 0.25, 100, 50, 5000.0) == pytest.approx(0.5, rel=1e-14)  # exponent 1/2
