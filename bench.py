@@ -183,7 +183,7 @@ def selection_outputs(W, N, dev):
             torch.zeros(2, dtype=torch.int32, device=dev))
 
 
-def setup_flat(cfg, dev, sgdb, seed):
+def setup_flat(cfg, dev, sgdb, seed, ema=False):
     """Workloads with one flat parameter vector (tiny SGD, Inception-sized RMSProp, large bf16 Adam)."""
     W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
     scales = wl.worker_scales(cfg.seed, W)
@@ -196,19 +196,27 @@ def setup_flat(cfg, dev, sgdb, seed):
     arr_d, tag_d = selection_sets(cfg, dev)
     opt = sgdb.Opt(**cfg.opt)
 
+    avg = theta.clone() if ema else None
+
     def step(i):
         opt.step = i + 1
-        sgdb.sgdb_step(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, mask, order, info)
+        if ema:  # the step plus the running average of the parameters (last line of the server's loop)
+            sgdb.sgdb_step_ema(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, avg, 0.9999,
+                               mask, order, info)
+        else:
+            sgdb.sgdb_step(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, mask, order, info)
 
     def check():
         assert info.cpu().tolist()[1] == 0, "a step reported a device-side error"
-        assert bool(torch.isfinite(theta).all())
+        assert bool(torch.isfinite(theta).all()) and (avg is None or bool(torch.isfinite(avg).all()))
 
     grad_bytes = N * P * grad.element_size()
     state = dict(grad=grad, theta=theta, s0=s0, s1=s1, opt=opt)
-    return dict(step=step, check=check, grad_bytes=grad_bytes, total_bytes=grad_bytes + 2 * (1 + n_state) * P * 4,
-                launches_per_step=1, kernel="stream_rows_kernel<%s, %s> (the step is this one launch)"
-                % (cfg.grad_dtype, cfg.opt["kind"]), state=state, extra={})
+    total = grad_bytes + 2 * (1 + n_state) * P * 4 + (2 * P * 4 if ema else 0)
+    return dict(step=step, check=check, grad_bytes=grad_bytes, total_bytes=total,
+                launches_per_step=1, kernel="stream_rows_kernel<%s, %s>%s (the step is this one launch)"
+                % (cfg.grad_dtype, cfg.opt["kind"], " + parameter average" if ema else ""), state=state,
+                extra={"parameter_average": True} if ema else {})
 
 
 def setup_segmented(cfg, dev, sgdb, seed):
@@ -355,7 +363,7 @@ def run_native(args, cfg):
     elif cfg.name.startswith("c4"):
         wk = setup_arrivals(cfg, dev, sgdb, seed)
     else:
-        wk = setup_flat(cfg, dev, sgdb, seed)
+        wk = setup_flat(cfg, dev, sgdb, seed, ema=args.ema)
     step = wk["step"]
 
     for i in range(args.warmup):
@@ -375,7 +383,7 @@ def run_native(args, cfg):
 
     # ---- end to end: gradients start in pinned host memory, new parameters are read back
     flat = not cfg.segments and not cfg.name.startswith("c4")
-    if args.no_e2e or not flat or cfg.W * cfg.P * (4 if cfg.grad_dtype == "f32" else 2) > 16e9:
+    if args.no_e2e or args.ema or not flat or cfg.W * cfg.P * (4 if cfg.grad_dtype == "f32" else 2) > 16e9:
         return finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, None, 0, clocks)
     W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
     st = wk["state"]
@@ -430,7 +438,7 @@ def finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_s
         peak, peak_kind = measured_hbm_peak()
         digest = kernel_source_digest()
         traffic = None
-        if (cfg.name == "c1_inception_rmsprop" and NCU_TRAFFIC["src_digest"] == digest
+        if (cfg.name == "c1_inception_rmsprop" and not args.ema and NCU_TRAFFIC["src_digest"] == digest
                 and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] is not None):
             traffic = NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] * total_bytes
         cpu = None
@@ -476,6 +484,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--workload", choices=["c0", "c1", "c2", "c3", "c4"], default="c1",
                     help="c1 (default) is the benchmark workload; the others time the remaining seeded workloads")
+    ap.add_argument("--ema", action="store_true",
+                    help="flat workloads: also keep the exponential moving average of the parameters (sgdb_step_ema)")
     ap.add_argument("--columns", type=int, default=0,
                     help="override P with a smaller column count (profiler captures); not the benchmark workload")
     args = ap.parse_args()

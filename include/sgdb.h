@@ -164,6 +164,40 @@ sgdb_status_t sgdb_step(const void *d_grad, sgdb_dtype_t dt, int64_t P, int64_t 
                         void *stream);
 
 /*
+ * sgdb_step_ema -- sgdb_step plus the line that follows the update in Algorithm 4:
+ * the exponential moving average of the parameters (Section 1.1),
+ *     avg <- alpha * avg + (1 - alpha) * theta(t),
+ * where theta(t) is the value of the parameters BEFORE this iteration's update, as
+ * Algorithm 4 writes it.  Same launch, 8 more bytes per parameter.
+ *   d_ema [P] fp32 in/out, 16-byte aligned.  The paper leaves the average before the
+ *   first iteration undefined; initialise d_ema with theta(0), so that it equals
+ *   theta(0) after iteration 0.  alpha in [0, 1] (the paper evaluates with 0.9999).
+ * When fewer than N gradients are current, d_ema is untouched like everything else.
+ */
+sgdb_status_t sgdb_step_ema(const void *d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld,
+                            const float *d_arrival, const int32_t *d_tags, int32_t t, int32_t N,
+                            int32_t b, float *d_theta, float *d_state0, float *d_state1,
+                            const sgdb_opt_t *opt, float *d_ema, float alpha, uint8_t *d_mask,
+                            int32_t *d_order, int32_t *d_info, void *stream);
+
+/*
+ * sgdb_ema -- the same average on its own, for callers of the separate calls
+ * (Algorithm 4's last line): avg <- alpha * avg + (1 - alpha) * theta.  Call it
+ * before sgdb_update to average the pre-update parameters as sgdb_step_ema does.
+ * d_info as in sgdb_aggregate.
+ */
+sgdb_status_t sgdb_ema(float *d_ema, const float *d_theta, int64_t P, float alpha,
+                       const int32_t *d_info, void *stream);
+
+/*
+ * sgdb_learning_rate -- the paper's learning-rate schedule (Appendix A.2, A.3), a host
+ * computation: gamma0 * beta^(t*N / (2*T)), with T = |X| / B the number of mini-batches
+ * in the data set.  N = number of aggregated workers for the synchronous rule; N = 1
+ * gives the asynchronous rule gamma0 * beta^(t / (2*T)).  NaN for T <= 0, N < 1 or t < 0.
+ */
+double sgdb_learning_rate(double gamma0, double beta, int64_t t, int64_t N, double T);
+
+/*
  * sgdb_step_segmented -- sgdb_step over a model stored as S separate tensors,
  * in one launch driven by a table in DEVICE memory (d_segments [S]).  One
  * selection serves all tensors, as one server iteration does in Algorithm 4.

@@ -24,7 +24,7 @@ _KINDS = {"sgd": SGDB_SGD, "momentum": SGDB_MOMENTUM, "rmsprop": SGDB_RMSPROP, "
 
 EXPORTS = (
     "sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented",
-    "sgdb_accumulate_arrival", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
+    "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
     "sgdb_set_tuning", "sgdb_strerror", "sgdb_version",
 )
 SGDB_STATIC_SCRATCH_BYTES = 8 << 20
@@ -79,6 +79,10 @@ def _load():
         "sgdb_aggregate": (i32, [vp, i32, i64, i64, i32, vp, vp, vp, vp]),
         "sgdb_update": (i32, [vp, vp, vp, vp, i64, ctypes.POINTER(_COpt), vp, vp]),
         "sgdb_step": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt), vp, vp, vp, vp]),
+        "sgdb_step_ema": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt), vp,
+                                ctypes.c_float, vp, vp, vp, vp]),
+        "sgdb_ema": (i32, [vp, vp, i64, ctypes.c_float, vp, vp]),
+        "sgdb_learning_rate": (ctypes.c_double, [ctypes.c_double, ctypes.c_double, i64, i64, ctypes.c_double]),
         "sgdb_step_segmented": (i32, [vp, i32, i32, vp, vp, i32, i32, i32, ctypes.POINTER(_COpt), vp, vp, vp, vp]),
         "sgdb_accumulate_arrival": (i32, [vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, ctypes.POINTER(_COpt), vp, vp]),
         "sgdb_step_host": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt),
@@ -184,6 +188,32 @@ def sgdb_step(grad, P: int, arrival, tags, t: int, N: int, b: int, theta, state0
                           _dev(state1, torch.float32, "state1"), ctypes.byref(c),
                           _dev(mask, torch.uint8, "mask"), _dev(order, torch.int32, "order"),
                           _dev(info, torch.int32, "info"), _stream(stream)), "sgdb_step")
+
+
+def sgdb_step_ema(grad, P: int, arrival, tags, t: int, N: int, b: int, theta, state0, state1, opt: Opt, ema,
+                  alpha: float, mask, order, info, ld: int | None = None, stream=None) -> None:
+    """sgdb_step plus avg <- alpha * avg + (1 - alpha) * theta(before the update), in the same launch."""
+    ld = grad.stride(0) if ld is None else ld
+    c = opt._c()
+    _check(_lib.sgdb_step_ema(_dev(grad, None, "grad"), _grad_dtype(grad), P, ld,
+                              _dev(arrival, torch.float32, "arrival"), _dev(tags, torch.int32, "tags"), t, N, b,
+                              _dev(theta, torch.float32, "theta"), _dev(state0, torch.float32, "state0"),
+                              _dev(state1, torch.float32, "state1"), ctypes.byref(c),
+                              _dev(ema, torch.float32, "ema"), alpha, _dev(mask, torch.uint8, "mask"),
+                              _dev(order, torch.int32, "order"), _dev(info, torch.int32, "info"), _stream(stream)),
+           "sgdb_step_ema")
+
+
+def sgdb_ema(ema, theta, alpha: float, info=None, P: int | None = None, stream=None) -> None:
+    """avg <- alpha * avg + (1 - alpha) * theta on its own."""
+    P = theta.numel() if P is None else P
+    _check(_lib.sgdb_ema(_dev(ema, torch.float32, "ema"), _dev(theta, torch.float32, "theta"), P, alpha,
+                         _dev(info, torch.int32, "info"), _stream(stream)), "sgdb_ema")
+
+
+def sgdb_learning_rate(gamma0: float, beta: float, t: int, N: int, T: float) -> float:
+    """gamma0 * beta^(t N / (2 T)): the paper's schedule (host computation)."""
+    return float(_lib.sgdb_learning_rate(gamma0, beta, t, N, T))
 
 
 def make_segment_table(segments, device) -> torch.Tensor:

@@ -293,10 +293,10 @@ sgdb_status_t sgdb_update(float* d_theta, float* d_state0, float* d_state1, cons
   return launch_status();
 }
 
-sgdb_status_t sgdb_step(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, const float* d_arrival,
-                        const int32_t* d_tags, int32_t t, int32_t N, int32_t b, float* d_theta,
-                        float* d_state0, float* d_state1, const sgdb_opt_t* opt, uint8_t* d_mask,
-                        int32_t* d_order, int32_t* d_info, void* stream) {
+static sgdb_status_t step_flat(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, const float* d_arrival,
+                               const int32_t* d_tags, int32_t t, int32_t N, int32_t b, float* d_theta,
+                               float* d_state0, float* d_state1, const sgdb_opt_t* opt, uint8_t* d_mask,
+                               int32_t* d_order, int32_t* d_info, float* d_ema, float alpha, void* stream) {
   sgdb_status_t st = check_selection_args(d_arrival, d_tags, N, b, d_mask, d_order, d_info);
   if (st != SGDB_OK) return st;
   st = check_flat(d_grad, dt, P, ld, N);
@@ -305,7 +305,8 @@ sgdb_status_t sgdb_step(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t 
   int ep = 0;
   st = prepare_rule(opt, d_state0, d_state1, &h, &ep);
   if (st != SGDB_OK) return st;
-  if (d_theta == nullptr || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
+  if (d_theta == nullptr || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1) ||
+      !is_aligned16(d_ema))
     return SGDB_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (P == 0) return launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
@@ -320,8 +321,50 @@ sgdb_status_t sgdb_step(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t 
   p.S = 1;
   p.N = N;
   set_in_kernel_selection(&p, d_arrival, d_tags, t, N + b, d_mask, d_order, d_info);
+  p.ema = d_ema;
+  p.ema_alpha = alpha;
+  p.ema_one_minus_alpha = static_cast<float>(1.0 - static_cast<double>(alpha));
   p.h = h;
   return launch_stream(dt, ep, p, tiles_of(dt, P), s);  // one launch: selection is the kernel's prologue
+}
+
+sgdb_status_t sgdb_step(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, const float* d_arrival,
+                        const int32_t* d_tags, int32_t t, int32_t N, int32_t b, float* d_theta,
+                        float* d_state0, float* d_state1, const sgdb_opt_t* opt, uint8_t* d_mask,
+                        int32_t* d_order, int32_t* d_info, void* stream) {
+  return step_flat(d_grad, dt, P, ld, d_arrival, d_tags, t, N, b, d_theta, d_state0, d_state1, opt, d_mask, d_order,
+                   d_info, nullptr, 0.0f, stream);
+}
+
+sgdb_status_t sgdb_step_ema(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, const float* d_arrival,
+                            const int32_t* d_tags, int32_t t, int32_t N, int32_t b, float* d_theta,
+                            float* d_state0, float* d_state1, const sgdb_opt_t* opt, float* d_ema, float alpha,
+                            uint8_t* d_mask, int32_t* d_order, int32_t* d_info, void* stream) {
+  if (d_ema == nullptr || !(alpha >= 0.0f && alpha <= 1.0f)) return SGDB_ERR_INVALID_ARG;
+  return step_flat(d_grad, dt, P, ld, d_arrival, d_tags, t, N, b, d_theta, d_state0, d_state1, opt, d_mask, d_order,
+                   d_info, d_ema, alpha, stream);
+}
+
+sgdb_status_t sgdb_ema(float* d_ema, const float* d_theta, int64_t P, float alpha, const int32_t* d_info,
+                       void* stream) {
+  if (d_ema == nullptr || d_theta == nullptr || P < 0 || !(alpha >= 0.0f && alpha <= 1.0f)) return SGDB_ERR_INVALID_ARG;
+  if (!is_aligned16(d_ema) || !is_aligned16(d_theta)) return SGDB_ERR_INVALID_ARG;
+  if (P == 0) return SGDB_OK;
+  const DeviceInfo* dev = nullptr;
+  sgdb_status_t st = device_info(&dev);
+  if (st != SGDB_OK) return st;
+  EmaParams p{d_ema, d_theta, P, alpha, static_cast<float>(1.0 - static_cast<double>(alpha)), d_info};
+  const long long chunks = (P + 3) / 4;
+  long long grid = (chunks + 255) / 256;
+  const long long cap = static_cast<long long>(dev->sms) * 8;
+  if (grid > cap) grid = cap;
+  ema_kernel<<<static_cast<unsigned>(grid), 256, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  return launch_status();
+}
+
+double sgdb_learning_rate(double gamma0, double beta, int64_t t, int64_t N, double T) {
+  if (!(T > 0.0) || N < 1 || t < 0) return std::nan("");
+  return gamma0 * std::pow(beta, static_cast<double>(t) * static_cast<double>(N) / (2.0 * T));
 }
 
 sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, sgdb_dtype_t dt,

@@ -211,6 +211,11 @@ __device__ __forceinline__ void apply_rule(const Hyper& h, float g, float& theta
   }
 }
 
+// Exponential moving average of the parameters: avg <- alpha * avg + (1 - alpha) * theta.
+__device__ __forceinline__ float ema_rule(float alpha, float one_minus_alpha, float avg, float theta) {
+  return __fmaf_rn(alpha, avg, __fmul_rn(one_minus_alpha, theta));
+}
+
 template <int EP>
 struct RuleTraits {
   static constexpr bool kTheta = EP != EP_MEAN;

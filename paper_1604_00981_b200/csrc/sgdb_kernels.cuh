@@ -132,6 +132,10 @@ struct StreamParams {
   uint8_t* mask_out;
   int32_t* order_out;
   int32_t* info_out;
+  // Optional (flat case): exponential moving average of the parameters, updated in the
+  // same pass from the value theta had BEFORE this step's update.
+  float* ema;
+  float ema_alpha, ema_one_minus_alpha;
   Hyper h;
 };
 
@@ -139,6 +143,7 @@ template <typename GT>
 struct TileDesc {
   const GT* grad;  // row 0 of this tile's columns
   float* theta;    // this tile's slice (mean output for EP_MEAN)
+  float* ema;      // this tile's slice of the averaged parameters, or nullptr
   float* s0;
   float* s1;
   long long ld;
@@ -176,8 +181,9 @@ __device__ __forceinline__ TileDesc<GT> locate_tile(const StreamParams& p, const
   const bool bulk_ok = ((reinterpret_cast<uintptr_t>(seg.grad) & 15u) == 0) &&
                        (((seg.ld * static_cast<long long>(sizeof(GT))) & 15) == 0);
   td.bulk_cols = bulk_ok ? (td.ncols / V) * V : 0;
+  td.ema = (p.ema != nullptr && p.table == nullptr) ? p.ema + col0 : nullptr;
   td.vec_ok = (((reinterpret_cast<uintptr_t>(seg.theta) | reinterpret_cast<uintptr_t>(seg.state0) |
-                 reinterpret_cast<uintptr_t>(seg.state1)) & 15u) == 0);
+                 reinterpret_cast<uintptr_t>(seg.state1) | reinterpret_cast<uintptr_t>(p.ema)) & 15u) == 0);
   return td;
 }
 
@@ -412,6 +418,13 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
             if (Rule::kTheta) load_floats<V>(td.theta + o, vec, n, th);
             if (Rule::kState0) load_floats<V>(td.s0 + o, vec, n, s0);
             if (Rule::kState1) load_floats<V>(td.s1 + o, vec, n, s1);
+            if (td.ema != nullptr) {
+              float avg[V];
+              load_floats<V>(td.ema + o, vec, n, avg);
+#pragma unroll
+              for (int e = 0; e < V; ++e) avg[e] = ema_rule(p.ema_alpha, p.ema_one_minus_alpha, avg[e], th[e]);
+              store_floats<V>(td.ema + o, vec, n, avg);
+            }
 #pragma unroll
             for (int e = 0; e < V; ++e) apply_rule<EP>(p.h, g[e], th[e], s0[e], s1[e]);
             store_floats<V>(td.theta + o, vec, n, th);
@@ -458,6 +471,34 @@ __global__ void __launch_bounds__(256) update_kernel(const UpdateParams p) {
     store_floats<4>(p.theta + i, vec, n, th);
     if (Rule::kState0) store_floats<4>(p.s0 + i, vec, n, s0);
     if (Rule::kState1) store_floats<4>(p.s1 + i, vec, n, s1);
+  }
+}
+
+// ====================================================================== parameter average alone
+
+struct EmaParams {
+  float* ema;
+  const float* theta;
+  long long P;
+  float alpha, one_minus_alpha;
+  const int32_t* info;
+};
+
+__global__ void __launch_bounds__(256) ema_kernel(const EmaParams p) {
+  if (p.info != nullptr && p.info[1] != SGDB_OK) return;
+  const long long chunks = (p.P + 3) / 4;
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  for (long long q = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; q < chunks; q += stride) {
+    const long long i = q * 4;
+    const long long rest = p.P - i;
+    const int n = rest < 4 ? static_cast<int>(rest) : 4;
+    const bool vec = n == 4;
+    float avg[4], th[4];
+    load_floats<4>(p.ema + i, vec, n, avg);
+    load_floats<4>(p.theta + i, vec, n, th);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) avg[e] = ema_rule(p.alpha, p.one_minus_alpha, avg[e], th[e]);
+    store_floats<4>(p.ema + i, vec, n, avg);
   }
 }
 

@@ -67,6 +67,17 @@ def test_host_checkable_errors_return_before_any_launch(lib):
     assert lib.sgdb_set_tuning(i32(0), i32(0)) == 0
 
 
+def test_learning_rate_schedule_is_a_host_computation(lib):
+    import oracle
+
+    lib.sgdb_learning_rate.restype = ctypes.c_double
+    lib.sgdb_learning_rate.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_int64, ctypes.c_int64, ctypes.c_double]
+    got = lib.sgdb_learning_rate(4.5, 0.94, 800, 100, 40_000.0)
+    assert abs(got - 4.5 * 0.94) < 1e-13 and abs(got - oracle.learning_rate(4.5, 0.94, 800, 100, 40_000.0)) < 1e-13
+    assert lib.sgdb_learning_rate(4.5, 0.94, 0, 100, 40_000.0) == 4.5
+    assert lib.sgdb_learning_rate(4.5, 0.94, 1, 0, 40_000.0) != lib.sgdb_learning_rate(4.5, 0.94, 1, 0, 40_000.0)  # NaN
+
+
 def test_optimizer_argument_checks(lib):
     from paper_1604_00981_b200.binding import _COpt
 

@@ -1,0 +1,84 @@
+"""Parity of the fused parameter average (sgdb_step_ema), the stand-alone average (sgdb_ema) and the
+learning-rate schedule with the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import (OPTS, TOL_BF16, TOL_F32, f32, gpu_opt, gpu_state, oracle_opt, oracle_state, rel_err,
+                     selection_buffers, step_inputs, to_dev)
+from paper_1604_00981_b200 import workload as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sgdb(cuda_device):
+    from paper_1604_00981_b200 import binding
+
+    return binding
+
+
+@pytest.mark.parametrize("kind,dtype,P,pad,alpha", [("rmsprop", "f32", 70_001, 3, 0.9999), ("sgd", "f32", 5, 0, 0.5),
+                                                    ("adam", "bf16", 70_003, 0, 0.9), ("momentum", "f32", 131_072, 0, 0.0),
+                                                    ("rmsprop", "bf16", 40_001, 7, 1.0)])
+def test_step_with_parameter_average(sgdb, cuda_device, kind, dtype, P, pad, alpha):
+    dev = cuda_device
+    W, N, T, seed = 20, 16, 5, 141
+    ld = P + pad
+    scales = wl.worker_scales(seed, W)
+    theta = wl.theta0(seed, P, dev)
+    avg = theta.clone()  # the average before the first iteration: theta(0)
+    s0, s1 = gpu_state(kind, P, dev)
+    twin = (theta.clone(), avg.clone()) + gpu_state(kind, P, dev)  # separate calls: sgdb_ema, then sgdb_step
+    th_o = theta.cpu().numpy().astype(np.float64)
+    avg_o = th_o.copy()
+    s0_o, s1_o = oracle_state(kind, P)
+    mask, order, info = selection_buffers(W, N, dev)
+    mask2, order2, info2 = selection_buffers(W, N, dev)
+    tol = TOL_F32 if dtype == "f32" else TOL_BF16
+    for t in range(T):
+        grad = wl.grad_matrix(seed, t, W, P, scales, dtype, dev, ld=ld, pad_value=float("nan"))
+        arrival, tags = step_inputs(seed, t, W, N)
+        a_d, t_d = to_dev(arrival, dev), to_dev(tags, dev)
+        sgdb.sgdb_step_ema(grad, P, a_d, t_d, t, N, W - N, theta, s0, s1, gpu_opt(OPTS[kind], t + 1), avg, alpha,
+                           mask, order, info, ld=ld)
+        rc, mask_o, order_o, n_valid = oracle.step_ema(wl.as_oracle_array(grad), P, arrival, tags, t, N, W - N, th_o,
+                                                       s0_o, s1_o, oracle_opt(OPTS[kind], t + 1), avg_o, f32(alpha), ld=ld)
+        assert rc == oracle.OK and info.cpu().tolist() == [n_valid, 0]
+        assert order.cpu().numpy().tolist() == order_o.tolist() and mask.cpu().numpy().tolist() == mask_o.tolist()
+        sgdb.sgdb_ema(twin[1], twin[0], alpha)
+        sgdb.sgdb_step(grad, P, a_d, t_d, t, N, W - N, twin[0], twin[2], twin[3], gpu_opt(OPTS[kind], t + 1),
+                       mask2, order2, info2, ld=ld)
+    assert rel_err(theta.cpu().numpy(), th_o) < tol
+    assert rel_err(avg.cpu().numpy(), avg_o) < tol
+    assert torch.equal(theta, twin[0]) and torch.equal(avg, twin[1])  # fused == separate, bit for bit
+
+
+def test_average_untouched_when_gradients_are_insufficient_and_bad_arguments(sgdb, cuda_device):
+    dev = cuda_device
+    W, N, P = 6, 5, 10_000
+    grad = torch.randn((W, P), device=dev)
+    theta, avg = torch.randn(P, device=dev), torch.randn(P, device=dev)
+    before = (theta.clone(), avg.clone())
+    mask, order, info = selection_buffers(W, N, dev)
+    arrival = to_dev(np.arange(W, dtype=np.float32), dev)
+    stale = to_dev(np.array([1, 1, 0, 0, 1, 1], np.int32), dev)
+    sgdb.sgdb_step_ema(grad, P, arrival, stale, 1, N, 1, theta, None, None, gpu_opt(OPTS["sgd"]), avg, 0.5, mask, order, info)
+    assert info.cpu().tolist() == [4, sgdb.SGDB_ERR_INSUFFICIENT]
+    assert torch.equal(theta, before[0]) and torch.equal(avg, before[1])
+    sgdb.sgdb_ema(avg, theta, 0.5, info)  # the separate call honours the same status word
+    assert torch.equal(avg, before[1])
+    for bad_alpha in (-0.1, 1.5, float("nan")):
+        with pytest.raises(sgdb.SgdbError):
+            sgdb.sgdb_step_ema(grad, P, arrival, stale, 1, N, 1, theta, None, None, gpu_opt(OPTS["sgd"]), avg, bad_alpha,
+                               mask, order, info)
+        with pytest.raises(sgdb.SgdbError):
+            sgdb.sgdb_ema(avg, theta, bad_alpha)
+
+
+def test_learning_rate_schedule_matches_oracle(sgdb):
+    for gamma0, beta, t, N, T in [(4.5, 0.94, 0, 100, 40_000.0), (4.5, 0.94, 12_345, 100, 40_036.0),
+                                  (0.045, 0.94, 777_777, 1, 40_036.0), (1e-4, 0.5, 3, 16, 12_500.0)]:
+        assert sgdb.sgdb_learning_rate(gamma0, beta, t, N, T) == pytest.approx(oracle.learning_rate(gamma0, beta, t, N, T), rel=1e-14)
+    assert np.isnan(sgdb.sgdb_learning_rate(1.0, 0.9, 1, 1, 0.0)) and np.isnan(sgdb.sgdb_learning_rate(1.0, 0.9, -1, 1, 5.0))
