@@ -84,6 +84,8 @@ def _load():
             "oracle_step",
             "oracle_accumulate_arrival",
             "oracle_step_ema",
+            "oracle_select_deadline",
+            "oracle_step_deadline",
         ):
             getattr(lib, name).restype = ctypes.c_int
         lib.oracle_ema.restype = None
@@ -199,6 +201,42 @@ def learning_rate(gamma0: float, beta: float, t: int, N: int, T: float) -> float
     """gamma0 * beta^(t N / (2 T)) (Appendix A.2, A.3)."""
     return float(_load().oracle_learning_rate(ctypes.c_double(gamma0), ctypes.c_double(beta), ctypes.c_int64(t),
                                               ctypes.c_int64(N), ctypes.c_double(T)))
+
+
+def select_deadline(arrival, tags, t: int, deadline: float, n_min: int = 1):
+    """Time-out rule: every gradient tagged t with arrival <= deadline.  Returns (status, mask, order[:n], n)."""
+    arrival = np.ascontiguousarray(arrival, dtype=np.float32)
+    tags = np.ascontiguousarray(tags, dtype=np.int32)
+    W = len(arrival)
+    mask = np.zeros(W, dtype=np.uint8)
+    order = np.full(W, -1, dtype=np.int32)
+    n = ctypes.c_int32(0)
+    rc = _load().oracle_select_deadline(_p(arrival), _p(tags), ctypes.c_int32(t), ctypes.c_int32(W),
+                                        ctypes.c_float(deadline), ctypes.c_int32(n_min), _p(mask), _p(order),
+                                        ctypes.byref(n))
+    return rc, mask, order[: n.value if rc == OK else 0], n.value
+
+
+def step_deadline(grad, P: int, arrival, tags, t: int, deadline: float, n_min: int, theta, s0, s1, opt: Opt,
+                  ld: int | None = None):
+    """One iteration with the time-out rule on fp64 theta/state (in place).  Returns (status, mask, order[:n], n)."""
+    g, dt = _grad(grad)
+    ld = g.shape[1] if ld is None else ld
+    arrival = np.ascontiguousarray(arrival, dtype=np.float32)
+    tags = np.ascontiguousarray(tags, dtype=np.int32)
+    W = len(arrival)
+    for a in (theta, s0, s1):
+        assert a is None or (a.dtype == np.float64 and a.flags.c_contiguous)
+    mask = np.zeros(W, dtype=np.uint8)
+    order = np.full(W, -1, dtype=np.int32)
+    n = ctypes.c_int32(0)
+    c = opt._c()
+    rc = _load().oracle_step_deadline(
+        _p(g), ctypes.c_int(dt), ctypes.c_int64(P), ctypes.c_int64(ld), _p(arrival), _p(tags), ctypes.c_int32(t),
+        ctypes.c_int32(W), ctypes.c_float(deadline), ctypes.c_int32(n_min), _p(theta), _p(s0), _p(s1),
+        ctypes.byref(c), _p(mask), _p(order), ctypes.byref(n),
+    )
+    return rc, mask, order[: n.value if rc == OK else 0], n.value
 
 
 def new_server_state():

@@ -102,6 +102,53 @@ int oracle_select(const float *arrival, const int32_t *tags, int32_t t, int32_t 
   return ORACLE_OK;
 }
 
+/*
+ * The alternative the paper names in its conclusion: a time-out instead of backup
+ * workers.  The paper gives no algorithm for it; the reading taken here is the direct
+ * counterpart of Algorithm 4: the server waits until `deadline`, keeps every gradient
+ * tagged t that has arrived by then (arrival <= deadline), drops the rest, and averages
+ * over the n it kept.  n_min >= 1 is the fewest it accepts; with fewer the iteration
+ * cannot complete and nothing changes.  PARITY UNPINNED BY THE PAPER (no definition
+ * printed); pinned by brute force and by its reductions to Algorithm 4.
+ *   mask [W], order [W] (first *n_kept entries used, arrival sequence), *n_kept.
+ */
+int oracle_select_deadline(const float *arrival, const int32_t *tags, int32_t t, int32_t W,
+                           float deadline, int32_t n_min, uint8_t *mask, int32_t *order,
+                           int32_t *n_kept) {
+  if (W < 1 || n_min < 1) return ORACLE_INVALID;
+  int32_t *seq = (int32_t *)malloc(sizeof(int32_t) * (size_t)W);
+  int32_t count = 0;
+  for (int32_t w = 0; w < W; ++w) {
+    if (tags[w] != t) continue;
+    if (!isfinite(arrival[w])) continue;
+    if (!(arrival[w] <= deadline)) continue; /* still on its way when the server stops waiting */
+    int32_t pos = count++;
+    while (pos > 0 && arrives_before(arrival, w, seq[pos - 1])) {
+      seq[pos] = seq[pos - 1];
+      --pos;
+    }
+    seq[pos] = w;
+  }
+  *n_kept = count;
+  if (count < n_min) {
+    free(seq);
+    return ORACLE_INSUFFICIENT;
+  }
+  for (int32_t w = 0; w < W; ++w) mask[w] = 0;
+  for (int32_t k = 0; k < count; ++k) {
+    order[k] = seq[k];
+    mask[seq[k]] = 1;
+  }
+  free(seq);
+  return ORACLE_OK;
+}
+
+/* One iteration with the time-out rule: mean over the n kept gradients, then the update. */
+int oracle_step_deadline(const void *grad, int dtype, int64_t P, int64_t ld, const float *arrival,
+                         const int32_t *tags, int32_t t, int32_t W, float deadline, int32_t n_min,
+                         double *theta, double *s0, double *s1, const oracle_opt_t *opt,
+                         uint8_t *mask, int32_t *order, int32_t *n_kept);
+
 /* Algorithm 4's update line, the part before the learning rate: (1/N) sum_{G in set} G. */
 int oracle_aggregate(const void *grad, int dtype, int64_t P, int64_t ld, int32_t N,
                      const int32_t *order, double *mean) {
@@ -166,6 +213,19 @@ int oracle_step(const void *grad, int dtype, int64_t P, int64_t ld, const float 
   if (rc != ORACLE_OK) return rc;
   double *mean = (double *)malloc(sizeof(double) * (size_t)(P > 0 ? P : 1));
   rc = oracle_aggregate(grad, dtype, P, ld, N, order, mean);
+  if (rc == ORACLE_OK) rc = oracle_update(theta, s0, s1, mean, P, opt);
+  free(mean);
+  return rc;
+}
+
+int oracle_step_deadline(const void *grad, int dtype, int64_t P, int64_t ld, const float *arrival,
+                         const int32_t *tags, int32_t t, int32_t W, float deadline, int32_t n_min,
+                         double *theta, double *s0, double *s1, const oracle_opt_t *opt,
+                         uint8_t *mask, int32_t *order, int32_t *n_kept) {
+  int rc = oracle_select_deadline(arrival, tags, t, W, deadline, n_min, mask, order, n_kept);
+  if (rc != ORACLE_OK) return rc;
+  double *mean = (double *)malloc(sizeof(double) * (size_t)(P > 0 ? P : 1));
+  rc = oracle_aggregate(grad, dtype, P, ld, *n_kept, order, mean); /* divisor: the number kept */
   if (rc == ORACLE_OK) rc = oracle_update(theta, s0, s1, mean, P, opt);
   free(mean);
   return rc;

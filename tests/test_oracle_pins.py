@@ -456,3 +456,67 @@ def test_learning_rate_schedule():
     assert oracle.learning_rate(4.5, 0.94, 1600, 100, T) == pytest.approx(4.5 * 0.94 ** 2, rel=1e-14)
     assert oracle.learning_rate(0.045, 0.94, 80_000, 1, T) == pytest.approx(0.045 * 0.94, rel=1e-14)  # asynchronous rule
     assert oracle.learning_rate(1.0, 0.25, 100, 50, 5000.0) == pytest.approx(0.5, rel=1e-14)  # exponent 1/2
+
+
+# ---------------------------------------------------------------- time-out instead of backup workers
+
+
+def test_deadline_selection_matches_replay_until_the_time_out():
+    """Replay: gradients reach the server in time order; at `deadline` it stops listening."""
+    rng = np.random.default_rng(21)
+    seen = set()
+    for trial in range(2000):
+        W = int(rng.integers(1, 9))
+        arrival, tags, t = _random_case(rng, W)
+        deadline = float(rng.choice([0.25, 0.5, 1.0, 1.25, 2.0, 7.0, 100.0, -0.5, np.inf]))
+        n_min = int(rng.integers(1, 4))
+        rc, mask, order, n = oracle.select_deadline(arrival, tags, t, deadline, n_min)
+        kept = []
+        for w in sorted((w for w in range(W) if math.isfinite(float(arrival[w]))), key=lambda w: (float(arrival[w]), w)):
+            if float(arrival[w]) > deadline:
+                break  # the server has stopped waiting
+            if int(tags[w]) == t:
+                kept.append(w)
+        assert n == len(kept)
+        if len(kept) < n_min:
+            assert rc == oracle.INSUFFICIENT and not mask.any()
+        else:
+            assert rc == oracle.OK and order.tolist() == kept
+            assert mask.tolist() == [1 if w in kept else 0 for w in range(W)]
+        seen.add(rc)
+    assert seen == {oracle.OK, oracle.INSUFFICIENT}
+
+
+def test_deadline_rule_reduces_to_algorithm4_and_divides_by_the_number_kept():
+    rng = np.random.default_rng(22)
+    W, N, P, t = 9, 6, 40, 3
+    arrival = rng.permutation(W).astype(np.float32) + 1.0  # distinct times 1..9
+    tags = np.full(W, t, np.int32)
+    grad = rng.normal(size=(W, P)).astype(np.float32)
+    # a deadline at the N-th arrival keeps exactly Algorithm 4's first N
+    rc, mask_n, order_n, _ = oracle.select(arrival, tags, t, N, W - N)
+    rc2, mask_d, order_d, n = oracle.select_deadline(arrival, tags, t, float(N), 1)
+    assert rc == rc2 == oracle.OK and n == N and order_d.tolist() == order_n.tolist() and mask_d.tolist() == mask_n.tolist()
+    th_a, th_b = np.zeros(P), np.zeros(P)
+    oracle.step(grad, P, arrival, tags, t, N, W - N, th_a, None, None, oracle.Opt(kind=oracle.SGD, lr=0.3))
+    oracle.step_deadline(grad, P, arrival, tags, t, float(N), 1, th_b, None, None, oracle.Opt(kind=oracle.SGD, lr=0.3))
+    assert th_a.tobytes() == th_b.tobytes()
+    # no deadline: plain synchronous SGD over every current gradient (library mean)
+    tags[4] = t - 1
+    th = np.zeros(P)
+    rc, mask, order, n = oracle.step_deadline(grad, P, arrival, tags, t, np.inf, 1, th, None, None,
+                                              oracle.Opt(kind=oracle.SGD, lr=1.0))
+    assert n == W - 1 and mask[4] == 0
+    np.testing.assert_allclose(th, -np.delete(grad, 4, axis=0).astype(np.float64).mean(axis=0), rtol=0, atol=1e-15)
+    # constant rows: the divisor is the number kept, whatever it is
+    consts = (2.0 ** np.arange(W)).astype(np.float32)
+    gc = np.repeat(consts[:, None], 3, axis=1)
+    for deadline in (1.0, 3.0, 8.0):
+        th = np.zeros(3)
+        rc, mask, order, n = oracle.step_deadline(gc, 3, arrival, tags, t, deadline, 1, th, None, None,
+                                                  oracle.Opt(kind=oracle.SGD, lr=1.0))
+        kept = [w for w in range(W) if arrival[w] <= deadline and tags[w] == t]
+        assert rc == oracle.OK and n == len(kept) and (th == -float(consts[kept].sum()) / len(kept)).all()
+    th = np.ones(3)
+    rc, *_ = oracle.step_deadline(gc, 3, arrival, tags, t, 0.5, 1, th, None, None, oracle.Opt(kind=oracle.SGD, lr=1.0))
+    assert rc == oracle.INSUFFICIENT and (th == 1).all()
