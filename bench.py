@@ -183,7 +183,7 @@ def selection_outputs(W, N, dev):
             torch.zeros(2, dtype=torch.int32, device=dev))
 
 
-def setup_flat(cfg, dev, sgdb, seed, ema=False):
+def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None):
     """Workloads with one flat parameter vector (tiny SGD, Inception-sized RMSProp, large bf16 Adam)."""
     W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
     scales = wl.worker_scales(cfg.seed, W)
@@ -197,10 +197,19 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False):
     opt = sgdb.Opt(**cfg.opt)
 
     avg = theta.clone() if ema else None
+    kept_mean = float(N)
+    if deadline is not None:  # time-out rule: the number of kept rows differs from draw to draw
+        order = torch.zeros(W, dtype=torch.int32, device=dev)
+        kept = [int(((wl.arrivals(cfg.seed, t, W) <= np.float32(deadline)) & (wl.tags(cfg.seed, t, W, N) == t)).sum())
+                for t in range(N_SETS)]
+        kept_mean = float(np.mean(kept))
 
     def step(i):
         opt.step = i + 1
-        if ema:  # the step plus the running average of the parameters (last line of the server's loop)
+        if deadline is not None:
+            sgdb.sgdb_step_deadline(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, deadline, 1, theta, s0, s1, opt,
+                                    mask, order, info)
+        elif ema:  # the step plus the running average of the parameters (last line of the server's loop)
             sgdb.sgdb_step_ema(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, avg, 0.9999,
                                mask, order, info)
         else:
@@ -210,13 +219,14 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False):
         assert info.cpu().tolist()[1] == 0, "a step reported a device-side error"
         assert bool(torch.isfinite(theta).all()) and (avg is None or bool(torch.isfinite(avg).all()))
 
-    grad_bytes = N * P * grad.element_size()
+    grad_bytes = int(kept_mean * P * grad.element_size())
     state = dict(grad=grad, theta=theta, s0=s0, s1=s1, opt=opt)
     total = grad_bytes + 2 * (1 + n_state) * P * 4 + (2 * P * 4 if ema else 0)
     return dict(step=step, check=check, grad_bytes=grad_bytes, total_bytes=total,
                 launches_per_step=1, kernel="stream_rows_kernel<%s, %s>%s (the step is this one launch)"
                 % (cfg.grad_dtype, cfg.opt["kind"], " + parameter average" if ema else ""), state=state,
-                extra={"parameter_average": True} if ema else {})
+                extra={"parameter_average": True} if ema else
+                ({"deadline_s": deadline, "mean_rows_kept": kept_mean} if deadline is not None else {}))
 
 
 def setup_segmented(cfg, dev, sgdb, seed):
@@ -363,7 +373,7 @@ def run_native(args, cfg):
     elif cfg.name.startswith("c4"):
         wk = setup_arrivals(cfg, dev, sgdb, seed)
     else:
-        wk = setup_flat(cfg, dev, sgdb, seed, ema=args.ema)
+        wk = setup_flat(cfg, dev, sgdb, seed, ema=args.ema, deadline=args.deadline)
     step = wk["step"]
 
     for i in range(args.warmup):
@@ -383,7 +393,7 @@ def run_native(args, cfg):
 
     # ---- end to end: gradients start in pinned host memory, new parameters are read back
     flat = not cfg.segments and not cfg.name.startswith("c4")
-    if args.no_e2e or args.ema or not flat or cfg.W * cfg.P * (4 if cfg.grad_dtype == "f32" else 2) > 16e9:
+    if args.no_e2e or args.ema or args.deadline is not None or not flat or cfg.W * cfg.P * (4 if cfg.grad_dtype == "f32" else 2) > 16e9:
         return finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, None, 0, clocks)
     W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
     st = wk["state"]
@@ -438,7 +448,7 @@ def finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_s
         peak, peak_kind = measured_hbm_peak()
         digest = kernel_source_digest()
         traffic = None
-        if (cfg.name == "c1_inception_rmsprop" and not args.ema and NCU_TRAFFIC["src_digest"] == digest
+        if (cfg.name == "c1_inception_rmsprop" and not args.ema and args.deadline is None and NCU_TRAFFIC["src_digest"] == digest
                 and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] is not None):
             traffic = NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] * total_bytes
         cpu = None
@@ -486,6 +496,8 @@ def main():
                     help="c1 (default) is the benchmark workload; the others time the remaining seeded workloads")
     ap.add_argument("--ema", action="store_true",
                     help="flat workloads: also keep the exponential moving average of the parameters (sgdb_step_ema)")
+    ap.add_argument("--deadline", type=float, default=None,
+                    help="flat workloads: time-out rule (sgdb_step_deadline) with this deadline in seconds")
     ap.add_argument("--columns", type=int, default=0,
                     help="override P with a smaller column count (profiler captures); not the benchmark workload")
     args = ap.parse_args()

@@ -198,6 +198,30 @@ sgdb_status_t sgdb_ema(float *d_ema, const float *d_theta, int64_t P, float alph
 double sgdb_learning_rate(double gamma0, double beta, int64_t t, int64_t N, double T);
 
 /*
+ * sgdb_select_deadline, sgdb_step_deadline -- the alternative the paper names in its
+ * conclusion (Section 6): a time-out instead of backup workers.  The paper prints no
+ * algorithm for it; this is Algorithm 4 with the stopping rule exchanged: the server
+ * listens until `deadline`, keeps EVERY gradient tagged t that arrived by then
+ * (arrival <= deadline, finite), drops the rest, and averages over the n it kept.
+ *
+ *   W            number of workers (rows of G, entries of d_arrival / d_tags / d_mask)
+ *   deadline     fp32 seconds, +infinity = wait for everyone; NaN is refused
+ *   n_min        1 <= n_min <= W: with fewer kept gradients the iteration does not
+ *                complete (d_info[1] = SGDB_ERR_INSUFFICIENT, nothing else is touched)
+ *   d_order [W]  out: the first n entries are the kept ids in arrival sequence
+ *   d_info  [2]  out: {n, status}; the mean divides by n
+ * sgdb_step_deadline is one launch, like sgdb_step.
+ */
+sgdb_status_t sgdb_select_deadline(const float *d_arrival, const int32_t *d_tags, int32_t t, int32_t W,
+                                   float deadline, int32_t n_min, uint8_t *d_mask, int32_t *d_order,
+                                   int32_t *d_info, void *stream);
+sgdb_status_t sgdb_step_deadline(const void *d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld,
+                                 const float *d_arrival, const int32_t *d_tags, int32_t t, int32_t W,
+                                 float deadline, int32_t n_min, float *d_theta, float *d_state0,
+                                 float *d_state1, const sgdb_opt_t *opt, uint8_t *d_mask,
+                                 int32_t *d_order, int32_t *d_info, void *stream);
+
+/*
  * sgdb_step_segmented -- sgdb_step over a model stored as S separate tensors,
  * in one launch driven by a table in DEVICE memory (d_segments [S]).  One
  * selection serves all tensors, as one server iteration does in Algorithm 4.

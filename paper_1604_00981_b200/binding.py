@@ -24,7 +24,7 @@ _KINDS = {"sgd": SGDB_SGD, "momentum": SGDB_MOMENTUM, "rmsprop": SGDB_RMSPROP, "
 
 EXPORTS = (
     "sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented",
-    "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
+    "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
     "sgdb_set_tuning", "sgdb_strerror", "sgdb_version",
 )
 SGDB_STATIC_SCRATCH_BYTES = 8 << 20
@@ -79,6 +79,9 @@ def _load():
         "sgdb_aggregate": (i32, [vp, i32, i64, i64, i32, vp, vp, vp, vp]),
         "sgdb_update": (i32, [vp, vp, vp, vp, i64, ctypes.POINTER(_COpt), vp, vp]),
         "sgdb_step": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt), vp, vp, vp, vp]),
+        "sgdb_select_deadline": (i32, [vp, vp, i32, i32, ctypes.c_float, i32, vp, vp, vp, vp]),
+        "sgdb_step_deadline": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, ctypes.c_float, i32, vp, vp, vp,
+                                     ctypes.POINTER(_COpt), vp, vp, vp, vp]),
         "sgdb_step_ema": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt), vp,
                                 ctypes.c_float, vp, vp, vp, vp]),
         "sgdb_ema": (i32, [vp, vp, i64, ctypes.c_float, vp, vp]),
@@ -188,6 +191,29 @@ def sgdb_step(grad, P: int, arrival, tags, t: int, N: int, b: int, theta, state0
                           _dev(state1, torch.float32, "state1"), ctypes.byref(c),
                           _dev(mask, torch.uint8, "mask"), _dev(order, torch.int32, "order"),
                           _dev(info, torch.int32, "info"), _stream(stream)), "sgdb_step")
+
+
+def sgdb_select_deadline(arrival, tags, t: int, deadline: float, n_min: int, mask, order, info, stream=None) -> None:
+    """Time-out rule: keep every gradient tagged t with arrival <= deadline.  order has W entries; info = {n, status}."""
+    W = arrival.numel()
+    _check(_lib.sgdb_select_deadline(_dev(arrival, torch.float32, "arrival"), _dev(tags, torch.int32, "tags"), t, W,
+                                     deadline, n_min, _dev(mask, torch.uint8, "mask"),
+                                     _dev(order, torch.int32, "order"), _dev(info, torch.int32, "info"),
+                                     _stream(stream)), "sgdb_select_deadline")
+
+
+def sgdb_step_deadline(grad, P: int, arrival, tags, t: int, deadline: float, n_min: int, theta, state0, state1,
+                       opt: Opt, mask, order, info, ld: int | None = None, stream=None) -> None:
+    """One fused iteration with the time-out rule: mean over the n gradients kept, then the optimizer rule."""
+    ld = grad.stride(0) if ld is None else ld
+    W = arrival.numel()
+    c = opt._c()
+    _check(_lib.sgdb_step_deadline(_dev(grad, None, "grad"), _grad_dtype(grad), P, ld,
+                                   _dev(arrival, torch.float32, "arrival"), _dev(tags, torch.int32, "tags"), t, W,
+                                   deadline, n_min, _dev(theta, torch.float32, "theta"),
+                                   _dev(state0, torch.float32, "state0"), _dev(state1, torch.float32, "state1"),
+                                   ctypes.byref(c), _dev(mask, torch.uint8, "mask"), _dev(order, torch.int32, "order"),
+                                   _dev(info, torch.int32, "info"), _stream(stream)), "sgdb_step_deadline")
 
 
 def sgdb_step_ema(grad, P: int, arrival, tags, t: int, N: int, b: int, theta, state0, state1, opt: Opt, ema,

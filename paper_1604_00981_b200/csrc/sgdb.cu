@@ -7,6 +7,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <limits>
 #include <mutex>
 
 #include "sgdb_kernels.cuh"
@@ -50,6 +51,8 @@ DeviceInfo g_dev[kMaxDevices];
 int g_stages = kDefaultStages;
 int g_ctas_per_sm = kDefaultCtasPerSm;
 int g_arrival_blocks_per_sm = 4;
+
+const float kNoDeadline = std::numeric_limits<float>::infinity();
 
 bool is_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -151,7 +154,8 @@ sgdb_status_t launch_stream_t(const StreamParams& p_in, long long total_tiles_hi
   auto kernel = stream_rows_kernel<GT, EP, kNT, kCH>;
 
   // shared memory: ring + 2 barriers per slot + order[N] + tile prefix[S + 1]
-  const size_t fixed = static_cast<size_t>((p.N + 3) & ~3) * 4 + (p.table ? (static_cast<size_t>(p.S) + 1) * 4 : 0) +
+  if (p.order_cap < p.N) p.order_cap = p.N;
+  const size_t fixed = static_cast<size_t>((p.order_cap + 3) & ~3) * 4 + (p.table ? (static_cast<size_t>(p.S) + 1) * 4 : 0) +
                        (p.arrival ? static_cast<size_t>(p.W) * 4 : 0) + 16;
   int ctas_per_sm = g_ctas_per_sm;
   int stages = g_stages;
@@ -205,7 +209,8 @@ sgdb_status_t launch_select(const float* d_arrival, const int32_t* d_tags, int32
                             uint8_t* d_mask, int32_t* d_order, int32_t* d_info, cudaStream_t stream) {
   const int W = N + b;
   const int threads = (W + 31) & ~31;  // one thread per worker
-  select_first_n_kernel<<<1, threads, 0, stream>>>(d_arrival, d_tags, t, N, W, d_mask, d_order, d_info);
+  select_first_n_kernel<<<1, threads, 0, stream>>>(d_arrival, d_tags, t, N, W, kNoDeadline, false, d_mask, d_order,
+                                                    d_info);
   return launch_status();
 }
 
@@ -218,6 +223,9 @@ void set_in_kernel_selection(StreamParams* p, const float* d_arrival, const int3
   p->tags = d_tags;
   p->t = t;
   p->W = W;
+  p->deadline = kNoDeadline;
+  p->keep_all = false;
+  p->order_cap = p->N;
   p->mask_out = d_mask;
   p->order_out = d_order;
   p->info_out = d_info;
@@ -365,6 +373,52 @@ sgdb_status_t sgdb_ema(float* d_ema, const float* d_theta, int64_t P, float alph
 double sgdb_learning_rate(double gamma0, double beta, int64_t t, int64_t N, double T) {
   if (!(T > 0.0) || N < 1 || t < 0) return std::nan("");
   return gamma0 * std::pow(beta, static_cast<double>(t) * static_cast<double>(N) / (2.0 * T));
+}
+
+sgdb_status_t sgdb_select_deadline(const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t W,
+                                   float deadline, int32_t n_min, uint8_t* d_mask, int32_t* d_order,
+                                   int32_t* d_info, void* stream) {
+  if (W < 1 || n_min < 1 || n_min > W || std::isnan(deadline)) return SGDB_ERR_INVALID_ARG;
+  sgdb_status_t st = check_selection_args(d_arrival, d_tags, W, 0, d_mask, d_order, d_info);
+  if (st != SGDB_OK) return st;
+  const int threads = (W + 31) & ~31;
+  select_first_n_kernel<<<1, threads, 0, static_cast<cudaStream_t>(stream)>>>(d_arrival, d_tags, t, n_min, W, deadline,
+                                                                              true, d_mask, d_order, d_info);
+  return launch_status();
+}
+
+sgdb_status_t sgdb_step_deadline(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, const float* d_arrival,
+                                 const int32_t* d_tags, int32_t t, int32_t W, float deadline, int32_t n_min,
+                                 float* d_theta, float* d_state0, float* d_state1, const sgdb_opt_t* opt,
+                                 uint8_t* d_mask, int32_t* d_order, int32_t* d_info, void* stream) {
+  if (W < 1 || n_min < 1 || n_min > W || std::isnan(deadline)) return SGDB_ERR_INVALID_ARG;
+  sgdb_status_t st = check_selection_args(d_arrival, d_tags, W, 0, d_mask, d_order, d_info);
+  if (st != SGDB_OK) return st;
+  st = check_flat(d_grad, dt, P, ld, n_min);
+  if (st != SGDB_OK) return st;
+  Hyper h;
+  int ep = 0;
+  st = prepare_rule(opt, d_state0, d_state1, &h, &ep);
+  if (st != SGDB_OK) return st;
+  if (d_theta == nullptr || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
+    return SGDB_ERR_INVALID_ARG;
+  if (P == 0) return sgdb_select_deadline(d_arrival, d_tags, t, W, deadline, n_min, d_mask, d_order, d_info, stream);
+  StreamParams p{};
+  p.table = nullptr;
+  p.flat.theta = d_theta;
+  p.flat.state0 = d_state0;
+  p.flat.state1 = d_state1;
+  p.flat.grad = d_grad;
+  p.flat.ld = ld;
+  p.flat.len = P;
+  p.S = 1;
+  p.N = n_min;
+  set_in_kernel_selection(&p, d_arrival, d_tags, t, W, d_mask, d_order, d_info);
+  p.deadline = deadline;
+  p.keep_all = true;
+  p.order_cap = W;
+  p.h = h;
+  return launch_stream(dt, ep, p, tiles_of(dt, P), static_cast<cudaStream_t>(stream));
 }
 
 sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, sgdb_dtype_t dt,

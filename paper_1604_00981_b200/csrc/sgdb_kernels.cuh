@@ -32,14 +32,16 @@ namespace sgdb {
 //
 //   s_key   [W] floats of shared memory, s_order [N] ints, s_count one int
 //   g_mask / g_order / g_info: global outputs, written only when `writer`
-// Returns true when at least N workers are valid; s_order is then filled.  When it
-// returns false nothing but g_info has been written.
-__device__ __forceinline__ bool block_select(const float* __restrict__ arrival,
-                                             const int32_t* __restrict__ tags, int32_t t, int32_t N,
-                                             int32_t W, float* s_key, int* s_order, int* s_count,
-                                             bool writer, uint8_t* __restrict__ g_mask,
-                                             int32_t* __restrict__ g_order,
-                                             int32_t* __restrict__ g_info) {
+// Time-out rule (keep_all): a worker is valid only if it also arrived by `deadline`,
+// and every valid worker is kept; N is then the fewest the caller accepts.
+// Returns the number of kept workers (s_order is filled with that many), or 0 when
+// fewer than N workers are valid; then nothing but g_info has been written.
+__device__ __forceinline__ int block_select(const float* __restrict__ arrival,
+                                            const int32_t* __restrict__ tags, int32_t t, int32_t N,
+                                            int32_t W, float deadline, bool keep_all, float* s_key,
+                                            int* s_order, int* s_count, bool writer,
+                                            uint8_t* __restrict__ g_mask, int32_t* __restrict__ g_order,
+                                            int32_t* __restrict__ g_info) {
   const int tid = threadIdx.x;
   const int nthreads = blockDim.x;
   if (tid == 0) *s_count = 0;
@@ -50,7 +52,7 @@ __device__ __forceinline__ bool block_select(const float* __restrict__ arrival,
     float a = 0.0f;
     if (w < W) {
       a = arrival[w];
-      valid = (tags[w] == t) && isfinite(a);
+      valid = (tags[w] == t) && isfinite(a) && (a <= deadline);
       s_key[w] = valid ? a : __int_as_float(0x7fc00000);
     }
     const unsigned votes = __ballot_sync(0xffffffffu, valid);
@@ -63,7 +65,8 @@ __device__ __forceinline__ bool block_select(const float* __restrict__ arrival,
     g_info[0] = n_valid;
     g_info[1] = enough ? SGDB_OK : SGDB_ERR_INSUFFICIENT;
   }
-  if (!enough) return false;
+  if (!enough) return 0;
+  const int keep = keep_all ? n_valid : N;
   for (int w = tid; w < W; w += nthreads) {
     const float a = s_key[w];
     int rank = 0;
@@ -72,7 +75,7 @@ __device__ __forceinline__ bool block_select(const float* __restrict__ arrival,
       const float aj = s_key[j];
       rank += ((aj < a) || (aj == a && j < w)) ? 1 : 0;
     }
-    const bool kept = (a == a) && rank < N;  // a != a: not valid
+    const bool kept = (a == a) && rank < keep;  // a != a: not valid
     if (kept) s_order[rank] = w;
     if (writer) {
       g_mask[w] = kept ? 1 : 0;
@@ -80,19 +83,20 @@ __device__ __forceinline__ bool block_select(const float* __restrict__ arrival,
     }
   }
   __syncthreads();
-  return true;
+  return keep;
 }
 
 __global__ void __launch_bounds__(1024) select_first_n_kernel(const float* __restrict__ arrival,
                                                               const int32_t* __restrict__ tags,
                                                               int32_t t, int32_t N, int32_t W,
+                                                              float deadline, bool keep_all,
                                                               uint8_t* __restrict__ mask,
                                                               int32_t* __restrict__ order,
                                                               int32_t* __restrict__ info) {
   __shared__ float s_key[SGDB_MAX_WORKERS];
   __shared__ int s_order[SGDB_MAX_WORKERS];
   __shared__ int s_count;
-  block_select(arrival, tags, t, N, W, s_key, s_order, &s_count, true, mask, order, info);
+  block_select(arrival, tags, t, N, W, deadline, keep_all, s_key, s_order, &s_count, true, mask, order, info);
 }
 
 // ====================================================================== row streaming
@@ -129,6 +133,9 @@ struct StreamParams {
   const int32_t* tags;
   int32_t t;
   int32_t W;
+  float deadline;   // time-out rule: arrival <= deadline (first-N rule: +infinity)
+  bool keep_all;    // time-out rule: keep every valid worker, N is the fewest accepted
+  int order_cap;    // ints of shared memory reserved for order[]: N, or W with keep_all
   uint8_t* mask_out;
   int32_t* order_out;
   int32_t* info_out;
@@ -203,18 +210,18 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int stages = p.stages;
-  const int N = p.N;
+  int N = p.N;  // rows to add; with the time-out rule the selection below decides it
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + static_cast<size_t>(stages) * STAGE_BYTES);
   uint64_t* empty_bar = full_bar + stages;
   int* order_s = reinterpret_cast<int*>(empty_bar + stages);
-  int* prefix_s = order_s + ((N + 3) & ~3);
+  int* prefix_s = order_s + ((p.order_cap + 3) & ~3);
   float* key_s = reinterpret_cast<float*>(prefix_s + (p.table != nullptr ? p.S + 1 : 0));
 
   if (p.arrival != nullptr) {
     // fewer than N current gradients: the iteration cannot complete, nothing is touched
-    if (!block_select(p.arrival, p.tags, p.t, N, p.W, key_s, order_s, &s_count, blockIdx.x == 0,
-                      p.mask_out, p.order_out, p.info_out))
-      return;
+    N = block_select(p.arrival, p.tags, p.t, N, p.W, p.deadline, p.keep_all, key_s, order_s, &s_count,
+                     blockIdx.x == 0, p.mask_out, p.order_out, p.info_out);
+    if (N == 0) return;
   } else {
     if (p.info != nullptr && p.info[1] != SGDB_OK) return;
     for (int i = tid; i < N; i += NT + 32) order_s[i] = p.order[i];
