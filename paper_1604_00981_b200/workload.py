@@ -81,14 +81,15 @@ def arrivals(seed: int, t: int, W: int) -> np.ndarray:
     return np.where(slow, 5.0 * a, a).astype(np.float32)
 
 
-def tags(seed: int, t: int, W: int, N: int) -> np.ndarray:
+def tags(seed: int, t: int, W: int, N: int, max_draws: int = 1_000_000) -> np.ndarray:
     """Iteration tag per worker: t, or t-1 with probability 0.1; redrawn while fewer than N are current."""
     g = _rng(seed, _S_TAG, t)
-    while True:
+    for _ in range(max_draws):
         stale = g.random(W) < 0.1
         tg = np.where(stale, t - 1, t).astype(np.int32)
         if int((tg == t).sum()) >= N:
             return tg
+    raise ValueError("no draw with %d current tags among %d workers at a stale rate of 0.1" % (N, W))
 
 
 def theta0(seed: int, P: int, device="cpu") -> torch.Tensor:

@@ -208,6 +208,33 @@ def test_accumulate_on_arrival(sgdb, cuda_device, kind, dtype, P, b):
         assert x is None or torch.equal(x, y)
 
 
+@pytest.mark.parametrize("kind,dtype", [("sgd", "f32"), ("rmsprop", "bf16")])
+def test_asynchronous_server_is_arrival_mode_with_n_equal_one(sgdb, cuda_device, kind, dtype):
+    """Algorithm 2 (the asynchronous parameter server) applies each gradient as it arrives.  That is the
+    arrival-by-arrival call with N = 1; gradients come from a delay queue, i.e. each was "computed" several
+    updates ago (simulated staleness), which changes nothing in what the server computes."""
+    dev = cuda_device
+    P, K, seed = 60_001, 12, 181
+    scales = wl.worker_scales(seed, K)
+    rows = wl.grad_matrix(seed, 0, K, P, scales, dtype, dev)
+    rows_h = wl.as_oracle_array(rows)
+    theta = wl.theta0(seed, P, dev)
+    s0, s1 = gpu_state(kind, P, dev)
+    th_o = theta.cpu().numpy().astype(np.float64)
+    s0_o, s1_o = oracle_state(kind, P)
+    acc = torch.empty(P, device=dev)
+    counter = torch.zeros(4, dtype=torch.int32, device=dev)
+    info = torch.zeros(2, dtype=torch.int32, device=dev)
+    queue = list(np.random.default_rng(seed).permutation(K))  # the order in which stale gradients surface
+    for step, w in enumerate(queue):
+        sgdb.sgdb_accumulate_arrival(rows[w], step, step, 1, acc, counter, theta, s0, s1, gpu_opt(OPTS[kind], step + 1), info)
+        assert info.cpu().tolist() == [2, 1]
+        mean = oracle.aggregate(rows_h, P, np.array([w], np.int32))  # the gradient itself
+        oracle.update(th_o, s0_o, s1_o, mean, oracle_opt(OPTS[kind], step + 1))
+    assert counter.cpu().tolist() == [0, K, 0, K]
+    assert rel_err(theta.cpu().numpy(), th_o) < (TOL_F32 if dtype == "f32" else TOL_BF16)
+
+
 # ------------------------------------------------------------------ gradients in host memory
 
 

@@ -196,6 +196,26 @@ def test_config3_shape_reduced_columns(sgdb, cuda_device):
 # ------------------------------------------------------------------ properties of the method
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_widest_server_1024_workers(sgdb, cuda_device, dtype):
+    """The largest accepted W: 880 kept of 1024 (about 920 carry the current tag), a ragged vector."""
+    _trajectory(sgdb, cuda_device, 1024, 880, 10_007, 2, dtype, OPTS["rmsprop"], seed=47, pad=1)
+
+
+def test_empty_parameter_vector_is_a_selection_only(sgdb, cuda_device):
+    dev = cuda_device
+    W, N = 10, 8
+    arrival, tags = step_inputs(49, 0, W, N)
+    mask, order, info = selection_buffers(W, N, dev)
+    grad = torch.zeros((W, 4), device=dev)
+    theta = torch.zeros(4, device=dev)
+    sgdb.sgdb_step(grad, 0, to_dev(arrival, dev), to_dev(tags, dev), 0, N, W - N, theta, None, None,
+                   gpu_opt(OPTS["sgd"]), mask, order, info, ld=4)
+    rc, mask_o, order_o, n_valid = oracle.select(arrival, tags, 0, N, W - N)
+    assert info.cpu().tolist() == [n_valid, 0] and order.cpu().numpy().tolist() == order_o.tolist()
+    assert mask.cpu().numpy().tolist() == mask_o.tolist() and (theta == 0).all()
+
+
 def test_fused_equals_separate_calls_bitwise(sgdb, cuda_device):
     dev = cuda_device
     W, N, P, seed = 30, 24, 123_457, 51

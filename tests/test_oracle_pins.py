@@ -520,3 +520,21 @@ def test_deadline_rule_reduces_to_algorithm4_and_divides_by_the_number_kept():
     th = np.ones(3)
     rc, *_ = oracle.step_deadline(gc, 3, arrival, tags, t, 0.5, 1, th, None, None, oracle.Opt(kind=oracle.SGD, lr=1.0))
     assert rc == oracle.INSUFFICIENT and (th == 1).all()
+
+
+# ---------------------------------------------------------------- the asynchronous server (Algorithm 2)
+
+
+def test_arrival_server_with_n_equal_one_is_algorithm2():
+    """Algorithm 2 applies every arriving gradient at once: theta <- theta - gamma G.  The arrival-by-arrival
+    server with N = 1 does exactly that; with SGD the result is theta0 - lr * (sum of all gradients)."""
+    rng = np.random.default_rng(31)
+    P, K, lr = 50, 17, 0.05
+    rows = rng.normal(size=(K, P)).astype(np.float32)
+    theta = rng.normal(size=P)
+    theta0 = theta.copy()
+    acc, state = np.zeros(P), oracle.new_server_state()
+    for k in range(K):
+        out = oracle.accumulate_arrival(rows[k], k, k, 1, acc, state, theta, None, None, oracle.Opt(kind=oracle.SGD, lr=lr))
+        assert out == 2 and state.tolist() == [0, k + 1, k + 1]
+    np.testing.assert_allclose(theta, theta0 - lr * rows.astype(np.float64).sum(axis=0), rtol=0, atol=1e-13)

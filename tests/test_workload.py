@@ -53,3 +53,10 @@ def test_segment_lengths_and_delivery_sequence():
     assert 30e6 < L.sum() < 100e6
     a = np.array([2.0, 1.0, np.inf, 1.0, 0.5], dtype=np.float32)
     assert wl.delivery_sequence(a).tolist() == [4, 1, 3, 0]
+
+
+def test_impossible_tag_request_raises_instead_of_looping():
+    import pytest
+
+    with pytest.raises(ValueError):
+        wl.tags(1, 0, 400, 400, max_draws=2000)  # all 400 current at a stale rate of 0.1: 0.9^400
