@@ -472,10 +472,20 @@ sgdb_status_t sgdb_accumulate_arrival(const void* d_row, sgdb_dtype_t dt, int32_
   if (row_tag != t || grid < 1) grid = 1;  // a wrongly tagged gradient only updates the bookkeeping
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const unsigned g = static_cast<unsigned>(grid);
-#define SGDB_ARRIVAL_CASE(EPV)                                                      \
-  case EPV:                                                                         \
-    if (dt == SGDB_BF16) accumulate_arrival_kernel<BF16, EPV><<<g, 256, 0, s>>>(p); \
-    else accumulate_arrival_kernel<float, EPV><<<g, 256, 0, s>>>(p);                \
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(g);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = SGDB_PDL ? 1 : 0;
+#define SGDB_ARRIVAL_CASE(EPV)                                                               \
+  case EPV:                                                                                  \
+    if (dt == SGDB_BF16) (void)cudaLaunchKernelEx(&cfg, accumulate_arrival_kernel<BF16, EPV>, p); \
+    else (void)cudaLaunchKernelEx(&cfg, accumulate_arrival_kernel<float, EPV>, p);                \
     break;
   switch (ep) {
     SGDB_ARRIVAL_CASE(EP_SGD)

