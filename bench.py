@@ -79,7 +79,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -454,9 +454,9 @@ def finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_s
         cpu = None
         if world == 1 and not args.no_cpu_baseline and cfg.name.startswith("c1"):
             P_sample = P // 4
-            sec, gbs = oracle_sample_run(cfg, P_sample, steps=10, warmup=1)
+            sec, gbs = oracle_sample_run(cfg, P_sample, steps=25, warmup=1)
             cpu = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
-                   "sample": "first %d of %d columns (1/4), all %d rows, 10 steps of %.2f s, single thread"
+                   "sample": "first %d of %d columns (1/4), all %d rows, 25 steps of %.2f s, single thread"
                              % (P_sample, P, W, sec)}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

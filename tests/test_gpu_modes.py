@@ -235,6 +235,70 @@ def test_asynchronous_server_is_arrival_mode_with_n_equal_one(sgdb, cuda_device,
     assert rel_err(theta.cpu().numpy(), th_o) < (TOL_F32 if dtype == "f32" else TOL_BF16)
 
 
+def test_two_level_aggregation_by_composition(sgdb, cuda_device):
+    """The paper's conclusion mentions combining the gradients of workers that share a machine before they
+    are sent.  With equal groups that is sgdb_aggregate per machine (its mean is what the machine sends,
+    when its slowest worker is done) followed by the server step over machines; the result is the mean over
+    all workers of the kept machines."""
+    dev = cuda_device
+    machines, per, keep, P, seed = 6, 4, 5, 50_001, 201
+    W = machines * per
+    grad = wl.grad_matrix(seed, 0, W, P, wl.worker_scales(seed, W), "f32", dev)
+    arrival_w = wl.arrivals(seed, 0, W)
+    arrival_m = arrival_w.reshape(machines, per).max(axis=1)
+    tags_m = np.zeros(machines, np.int32)
+    ld = (P + 3) // 4 * 4  # machine rows start on 16-byte boundaries
+    sent = torch.zeros((machines, ld), device=dev)
+    ok = to_dev(np.array([per, 0], np.int32), dev)
+    for m in range(machines):
+        ids = to_dev(np.arange(m * per, (m + 1) * per, dtype=np.int32), dev)
+        sgdb.sgdb_aggregate(grad, P, per, ids, ok, sent[m, :P])
+    theta = wl.theta0(seed, P, dev)
+    th_o = theta.cpu().numpy().astype(np.float64)
+    mask, order, info = selection_buffers(machines, keep, dev)
+    sgdb.sgdb_step(sent, P, to_dev(arrival_m, dev), to_dev(tags_m, dev), 0, keep, machines - keep, theta, None, None,
+                   gpu_opt(OPTS["sgd"]), mask, order, info, ld=ld)
+    rc, mask_o, order_o, _ = oracle.select(arrival_m, tags_m, 0, keep, machines - keep)
+    assert rc == oracle.OK and order.cpu().numpy().tolist() == order_o.tolist()
+    workers = np.concatenate([np.arange(m * per, (m + 1) * per) for m in order_o]).astype(np.int32)
+    mean = oracle.aggregate(wl.as_oracle_array(grad), P, workers)  # flat mean over the 20 workers of the kept machines
+    oracle.update(th_o, None, None, mean, oracle_opt(OPTS["sgd"]))
+    assert rel_err(theta.cpu().numpy(), th_o) < TOL_F32
+
+
+def test_checkpoint_and_resume_is_bit_identical(sgdb, cuda_device):
+    """All state lives in the caller's buffers (parameters, optimizer state, accumulator, server counters):
+    copying them out in the middle of an iteration and carrying on from the copies changes no bit."""
+    dev = cuda_device
+    N, b, P, seed, kind = 10, 2, 30_001, 191, "adam"
+    W = N + b
+    scales = wl.worker_scales(seed, W)
+
+    def fresh():
+        return dict(theta=wl.theta0(seed, P, dev), s0=torch.zeros(P, device=dev), s1=torch.zeros(P, device=dev),
+                    acc=torch.zeros(P, device=dev), counter=torch.zeros(4, dtype=torch.int32, device=dev))
+
+    def deliver(st, t, ids, grad, tags):
+        info = torch.zeros(2, dtype=torch.int32, device=dev)
+        for w in ids:
+            sgdb.sgdb_accumulate_arrival(grad[w], int(tags[w]), t, N, st["acc"], st["counter"], st["theta"], st["s0"],
+                                         st["s1"], gpu_opt(OPTS[kind], t + 1), info)
+
+    straight, resumed = fresh(), fresh()
+    for t in range(3):
+        grad = wl.grad_matrix(seed, t, W, P, scales, "bf16", dev)
+        arrival, tags = step_inputs(seed, t, W, N)
+        ids = wl.delivery_sequence(arrival).tolist()
+        deliver(straight, t, ids, grad, tags)
+        deliver(resumed, t, ids[:5], grad, tags)  # stop in the middle of the iteration ...
+        saved = {k: v.cpu().clone() for k, v in resumed.items()}
+        resumed = {k: v.to(dev) for k, v in saved.items()}  # ... and carry on from the copies, in new buffers
+        deliver(resumed, t, ids[5:], grad, tags)
+    for k in straight:
+        assert torch.equal(straight[k], resumed[k]), k
+    assert straight["counter"].cpu().tolist() == [0, 3 * W, 0, 3]
+
+
 # ------------------------------------------------------------------ gradients in host memory
 
 
