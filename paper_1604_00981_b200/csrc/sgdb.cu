@@ -287,7 +287,7 @@ sgdb_status_t sgdb_update(float* d_theta, float* d_state0, float* d_state1, cons
   if (st != SGDB_OK) return st;
   UpdateParams p{d_theta, d_state0, d_state1, d_mean, P, d_info, h};
   const long long chunks = (P + 3) / 4;
-  long long grid = (chunks + 255) / 256;
+  long long grid = (chunks + 2 * 256 - 1) / (2 * 256);  // two chunks per thread and pass
   const long long cap = static_cast<long long>(dev->sms) * 8;
   if (grid > cap) grid = cap;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

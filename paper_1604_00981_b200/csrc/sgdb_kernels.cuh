@@ -469,21 +469,36 @@ __global__ void __launch_bounds__(256) update_kernel(const UpdateParams p) {
   if (p.info != nullptr && p.info[1] != SGDB_OK) return;
   const long long chunks = (p.P + 3) / 4;
   const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-  for (long long q = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; q < chunks; q += stride) {
-    const long long i = q * 4;
-    const long long rest = p.P - i;
-    const int n = rest < 4 ? static_cast<int>(rest) : 4;
-    const bool vec = n == 4;
-    float g[4], th[4], s0[4], s1[4];
-    load_floats<4>(p.mean + i, vec, n, g);
-    load_floats<4>(p.theta + i, vec, n, th);
-    if (Rule::kState0) load_floats<4>(p.s0 + i, vec, n, s0);
-    if (Rule::kState1) load_floats<4>(p.s1 + i, vec, n, s1);
+  constexpr int U = 2;  // two chunks per thread and pass, all loads issued before the arithmetic
+  for (long long q0 = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; q0 < chunks; q0 += stride * U) {
+    float g[U][4], th[U][4], s0[U][4], s1[U][4];
+    int n[U];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) apply_rule<EP>(p.h, g[e], th[e], s0[e], s1[e]);
-    store_floats<4>(p.theta + i, vec, n, th);
-    if (Rule::kState0) store_floats<4>(p.s0 + i, vec, n, s0);
-    if (Rule::kState1) store_floats<4>(p.s1 + i, vec, n, s1);
+    for (int u = 0; u < U; ++u) {
+      const long long q = q0 + u * stride;
+      const long long i = q * 4;
+      const long long rest = p.P - i;
+      n[u] = q < chunks ? (rest < 4 ? static_cast<int>(rest) : 4) : 0;
+      if (n[u] > 0) {
+        const bool vec = n[u] == 4;
+        load_floats<4>(p.mean + i, vec, n[u], g[u]);
+        load_floats<4>(p.theta + i, vec, n[u], th[u]);
+        if (Rule::kState0) load_floats<4>(p.s0 + i, vec, n[u], s0[u]);
+        if (Rule::kState1) load_floats<4>(p.s1 + i, vec, n[u], s1[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (n[u] > 0) {
+        const long long i = (q0 + u * stride) * 4;
+        const bool vec = n[u] == 4;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) apply_rule<EP>(p.h, g[u][e], th[u][e], s0[u][e], s1[u][e]);
+        store_floats<4>(p.theta + i, vec, n[u], th[u]);
+        if (Rule::kState0) store_floats<4>(p.s0 + i, vec, n[u], s0[u]);
+        if (Rule::kState1) store_floats<4>(p.s1 + i, vec, n[u], s1[u]);
+      }
+    }
   }
 }
 
