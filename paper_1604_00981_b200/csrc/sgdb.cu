@@ -231,6 +231,21 @@ void set_in_kernel_selection(StreamParams* p, const float* d_arrival, const int3
   p->info_out = d_info;
 }
 
+// Parameters of the row-streaming kernel for one flat vector; selection fields are filled in by the caller.
+StreamParams flat_params(float* theta, float* state0, float* state1, const void* grad, int64_t ld, int64_t P, int32_t N) {
+  StreamParams p{};
+  p.table = nullptr;
+  p.flat.theta = theta;
+  p.flat.state0 = state0;
+  p.flat.state1 = state1;
+  p.flat.grad = grad;
+  p.flat.ld = ld;
+  p.flat.len = P;
+  p.S = 1;
+  p.N = N;
+  return p;
+}
+
 sgdb_status_t check_flat(const void* grad, int dt, int64_t P, int64_t ld, int32_t N) {
   if (grad == nullptr || !dtype_ok(dt)) return SGDB_ERR_INVALID_ARG;
   if (P < 0 || ld < P || N < 1 || N > SGDB_MAX_WORKERS) return SGDB_ERR_INVALID_ARG;
@@ -258,17 +273,9 @@ sgdb_status_t sgdb_aggregate(const void* d_grad, sgdb_dtype_t dt, int64_t P, int
   if (st != SGDB_OK) return st;
   if (d_order == nullptr || d_mean == nullptr || !is_aligned16(d_mean)) return SGDB_ERR_INVALID_ARG;
   if (P == 0) return SGDB_OK;
-  StreamParams p{};
-  p.table = nullptr;
-  p.flat.theta = d_mean;
-  p.flat.grad = d_grad;
-  p.flat.ld = ld;
-  p.flat.len = P;
-  p.S = 1;
-  p.N = N;
+  StreamParams p = flat_params(d_mean, nullptr, nullptr, d_grad, ld, P, N);  // the mean goes where theta would
   p.order = d_order;
   p.info = d_info;
-  p.status_out = nullptr;
   return launch_stream(dt, EP_MEAN, p, tiles_of(dt, P), static_cast<cudaStream_t>(stream));
 }
 
@@ -318,16 +325,7 @@ static sgdb_status_t step_flat(const void* d_grad, sgdb_dtype_t dt, int64_t P, i
     return SGDB_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (P == 0) return launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
-  StreamParams p{};
-  p.table = nullptr;
-  p.flat.theta = d_theta;
-  p.flat.state0 = d_state0;
-  p.flat.state1 = d_state1;
-  p.flat.grad = d_grad;
-  p.flat.ld = ld;
-  p.flat.len = P;
-  p.S = 1;
-  p.N = N;
+  StreamParams p = flat_params(d_theta, d_state0, d_state1, d_grad, ld, P, N);
   set_in_kernel_selection(&p, d_arrival, d_tags, t, N + b, d_mask, d_order, d_info);
   p.ema = d_ema;
   p.ema_alpha = alpha;
@@ -403,16 +401,7 @@ sgdb_status_t sgdb_step_deadline(const void* d_grad, sgdb_dtype_t dt, int64_t P,
   if (d_theta == nullptr || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
     return SGDB_ERR_INVALID_ARG;
   if (P == 0) return sgdb_select_deadline(d_arrival, d_tags, t, W, deadline, n_min, d_mask, d_order, d_info, stream);
-  StreamParams p{};
-  p.table = nullptr;
-  p.flat.theta = d_theta;
-  p.flat.state0 = d_state0;
-  p.flat.state1 = d_state1;
-  p.flat.grad = d_grad;
-  p.flat.ld = ld;
-  p.flat.len = P;
-  p.S = 1;
-  p.N = n_min;
+  StreamParams p = flat_params(d_theta, d_state0, d_state1, d_grad, ld, P, n_min);
   set_in_kernel_selection(&p, d_arrival, d_tags, t, W, d_mask, d_order, d_info);
   p.deadline = deadline;
   p.keep_all = true;
@@ -570,16 +559,7 @@ sgdb_status_t sgdb_step_host(const void* h_grad, sgdb_dtype_t dt, int64_t P, int
                           static_cast<size_t>(P) * esize, cudaMemcpyHostToDevice, s) != cudaSuccess)
         return launch_status();
     }
-    StreamParams p{};
-    p.table = nullptr;
-    p.flat.theta = d_theta;
-    p.flat.state0 = d_state0;
-    p.flat.state1 = d_state1;
-    p.flat.grad = d_rows;
-    p.flat.ld = pitch;
-    p.flat.len = P;
-    p.S = 1;
-    p.N = N;
+    StreamParams p = flat_params(d_theta, d_state0, d_state1, d_rows, pitch, P, N);
     p.order = d_order;
     p.info = d_info;
     p.status_out = d_info + 1;
