@@ -105,6 +105,27 @@ def test_aggregate_matches_oracle(sgdb, cuda_device, dtype, P, pad):
     assert np.array_equal(got[:P], acc / np.float32(N))
 
 
+def test_aggregate_error_within_the_sequential_sum_bound(sgdb, cuda_device):
+    """A sequential fp32 sum of N terms is off by at most (N - 1) u sum|g_k| (u = 2^-24), the division adds
+    one more rounding: every element of the device mean must sit inside that band around the fp64 mean."""
+    dev = cuda_device
+    c = wl.CONFIGS[1]
+    W, N, P = c.W, c.N, 300_007
+    grad = wl.grad_matrix(c.seed, 0, W, P, wl.worker_scales(c.seed, W), "f32", dev)
+    arrival, tags = step_inputs(c.seed, 0, W, N)
+    rc, _, order_o, _ = oracle.select(arrival, tags, 0, N, W - N)
+    mean = torch.empty(P, device=dev)
+    sgdb.sgdb_aggregate(grad, P, N, to_dev(order_o, dev), None, mean)
+    rows = wl.as_oracle_array(grad)[order_o].astype(np.float64)
+    ref = rows.mean(axis=0)
+    u = 2.0 ** -24
+    bound = ((N - 1) * u * np.abs(rows).sum(axis=0)) / N + u * np.abs(ref) + 1e-45
+    err = np.abs(mean.cpu().numpy().astype(np.float64) - ref)
+    assert (err <= bound).all()
+    assert err.max() > 0  # it is an fp32 sum, not the oracle in disguise
+    assert rel_err(mean.cpu().numpy(), ref) < TOL_F32 / 5
+
+
 def test_aggregate_skipped_when_selection_failed(sgdb, cuda_device):
     P = 5000
     grad = torch.ones((3, P), device=cuda_device)
