@@ -225,7 +225,10 @@ sgdb_status_t sgdb_step_deadline(const void *d_grad, sgdb_dtype_t dt, int64_t P,
  * sgdb_step_segmented -- sgdb_step over a model stored as S separate tensors,
  * in one launch driven by a table in DEVICE memory (d_segments [S]).  One
  * selection serves all tensors, as one server iteration does in Algorithm 4.
- * S <= SGDB_MAX_SEGMENTS, otherwise SGDB_ERR_UNSUPPORTED.
+ * S <= SGDB_MAX_SEGMENTS, otherwise SGDB_ERR_UNSUPPORTED.  The table cannot be
+ * inspected from the host: a segment with a null theta or grad pointer, or without a
+ * state pointer its rule needs, is skipped by the kernel and d_info[1] then reads
+ * SGDB_ERR_INVALID_ARG (the other segments are still updated).
  */
 sgdb_status_t sgdb_step_segmented(const sgdb_segment_t *d_segments, int32_t S, sgdb_dtype_t dt,
                                   const float *d_arrival, const int32_t *d_tags, int32_t t,

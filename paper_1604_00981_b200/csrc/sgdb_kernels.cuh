@@ -163,9 +163,10 @@ struct TileDesc {
   int ncols;      // valid columns in the tile
   int bulk_cols;  // leading columns delivered by bulk copy (0: none)
   bool vec_ok;    // theta/state slices may be accessed 16 bytes at a time
+  bool bad;       // a pointer this rule needs is null in the segment table: the tile is skipped
 };
 
-template <typename GT, int TILE>
+template <typename GT, int TILE, int EP>
 __device__ __forceinline__ TileDesc<GT> locate_tile(const StreamParams& p, const int* prefix_s,
                                                     int tile) {
   constexpr int V = GradTraits<GT>::kVec;
@@ -194,9 +195,19 @@ __device__ __forceinline__ TileDesc<GT> locate_tile(const StreamParams& p, const
   const bool bulk_ok = ((reinterpret_cast<uintptr_t>(seg.grad) & 15u) == 0) &&
                        (((seg.ld * static_cast<long long>(sizeof(GT))) & 15) == 0);
   td.bulk_cols = bulk_ok ? (td.ncols / V) * V : 0;
+  td.bad = false;
   td.ema = (p.ema != nullptr && p.table == nullptr) ? p.ema + col0 : nullptr;
   td.vec_ok = (((reinterpret_cast<uintptr_t>(seg.theta) | reinterpret_cast<uintptr_t>(seg.state0) |
                  reinterpret_cast<uintptr_t>(seg.state1) | reinterpret_cast<uintptr_t>(p.ema)) & 15u) == 0);
+  // The table lives in device memory, so the host cannot check it: a segment without a
+  // pointer its rule needs is left alone (and reported) instead of being dereferenced.
+  using Rule = RuleTraits<EP>;
+  if (seg.theta == nullptr || seg.grad == nullptr || (Rule::kState0 && seg.state0 == nullptr) ||
+      (Rule::kState1 && seg.state1 == nullptr)) {
+    td.bad = true;
+    td.ncols = 0;
+    td.bulk_cols = 0;
+  }
   return td;
 }
 
@@ -278,7 +289,7 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
       int s = 0;
       uint32_t phase = 0;
       for (int tile = blockIdx.x; tile < total_tiles && !timed_out; tile += gridDim.x) {
-        const TileDesc<GT> td = locate_tile<GT, TILE>(p, prefix_s, tile);
+        const TileDesc<GT> td = locate_tile<GT, TILE, EP>(p, prefix_s, tile);
         if (td.bulk_cols == 0) continue;
         const uint32_t bytes = static_cast<uint32_t>(td.bulk_cols) * sizeof(GT);
         for (int k = 0; k < N; ++k) {
@@ -303,7 +314,7 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
     int s = 0;
     uint32_t phase = 0;
     for (int tile = blockIdx.x; tile < total_tiles && !timed_out; tile += gridDim.x) {
-      const TileDesc<GT> td = locate_tile<GT, TILE>(p, prefix_s, tile);
+      const TileDesc<GT> td = locate_tile<GT, TILE, EP>(p, prefix_s, tile);
 
       float acc[CH][V];
 #pragma unroll
@@ -327,6 +338,10 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
       };
       const bool has_tail = td.bulk_cols < td.ncols;
 
+      if (td.bad) {
+        if (tid == 0 && p.status_out != nullptr) *p.status_out = SGDB_ERR_INVALID_ARG;
+        continue;
+      }
       if (td.bulk_cols == 0) {
         for (int k = 0; k < N; ++k) add_row_tail(k);
       } else {

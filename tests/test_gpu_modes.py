@@ -132,6 +132,15 @@ def test_segmented_edge_cases(sgdb, cuda_device):
         sgdb.sgdb_step_segmented(keep, sgdb.SGDB_MAX_SEGMENTS + 1, torch.float32, a_d, t_d, 0, N, 1,
                                  gpu_opt(OPTS["sgd"]), mask, order, info)
     assert e.value.status == sgdb.SGDB_ERR_UNSUPPORTED
+    # a segment without the state its rule needs is skipped and reported, never dereferenced
+    th = [torch.zeros(5000, device=dev) for _ in range(3)]
+    vel = [torch.zeros(5000, device=dev), None, torch.zeros(5000, device=dev)]
+    gr = [torch.ones((W, 5000), device=dev) for _ in range(3)]
+    table = sgdb.make_segment_table([(th[i], vel[i], None, gr[i]) for i in range(3)], dev)
+    sgdb.sgdb_step_segmented(table, 3, torch.float32, a_d, t_d, 0, N, 1, gpu_opt(dict(kind="momentum", lr=1.0, momentum=0.5)),
+                             mask, order, info)
+    assert info.cpu().tolist() == [4, sgdb.SGDB_ERR_INVALID_ARG]
+    assert (th[0] == -1).all() and (th[1] == 0).all() and (th[2] == -1).all()
     # the largest table, every tensor tiny
     S = sgdb.SGDB_MAX_SEGMENTS
     theta = torch.zeros(S * 3, device=dev)
