@@ -219,6 +219,31 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None):
         assert info.cpu().tolist()[1] == 0, "a step reported a device-side error"
         assert bool(torch.isfinite(theta).all()) and (avg is None or bool(torch.isfinite(avg).all()))
 
+    def graph_replay():
+        """Launch-bound sizes: the same steps captured once in a CUDA graph and replayed, so that the host's
+        per-call cost (Python, ctypes, launch) is out of the picture."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(3):
+                step(i)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(N_SETS):
+                step(i)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        for _ in range(20):
+            graph.replay()
+        stop.record()
+        torch.cuda.synchronize()
+        return {"cuda_graph_replay_us_per_step": 1e3 * start.elapsed_time(stop) / (20 * N_SETS)}
+
     grad_bytes = int(kept_mean * P * grad.element_size())
     state = dict(grad=grad, theta=theta, s0=s0, s1=s1, opt=opt)
     total = grad_bytes + 2 * (1 + n_state) * P * 4 + (2 * P * 4 if ema else 0)
@@ -226,7 +251,8 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None):
                 launches_per_step=1, kernel="stream_rows_kernel<%s, %s>%s (the step is this one launch)"
                 % (cfg.grad_dtype, cfg.opt["kind"], " + parameter average" if ema else ""), state=state,
                 extra={"parameter_average": True} if ema else
-                ({"deadline_s": deadline, "mean_rows_kept": kept_mean} if deadline is not None else {}))
+                ({"deadline_s": deadline, "mean_rows_kept": kept_mean} if deadline is not None else
+                 (graph_replay if P * W <= 1_000_000 else {})))
 
 
 def setup_segmented(cfg, dev, sgdb, seed):
@@ -464,8 +490,11 @@ def finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_s
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": cfg.name, "P": P, "W": W, "N": N, "b": b, "optimizer": cfg.opt["kind"],
                        "grad_dtype": cfg.grad_dtype, "sharding": "one parameter-server column shard of P per GPU",
-                       "l2": "inputs larger than L2 (126 MB): %.3f GB of gradient rows and %.1f MB of parameters and "
-                             "state per step" % (grad_bytes / 1e9, (total_bytes - grad_bytes) / 2e6)},
+                       "l2": ("inputs larger than L2 (126 MB): %.3f GB of gradient rows and %.1f MB of parameters and "
+                              "state per step" % (grad_bytes / 1e9, (total_bytes - grad_bytes) / 2e6))
+                             if total_bytes > 4 * 126e6 else
+                             "inputs fit in L2 (%.0f KB per step): a launch-bound workload, read its step time only"
+                             % (total_bytes / 1e3)},
             "step_us": ms_per_step * 1e3,
             "total_gbs_per_gpu": total_gbs_per_gpu,
             "pct_of_nominal_8tbs": 100.0 * total_gbs_per_gpu / NOMINAL_HBM_GBS,
