@@ -202,6 +202,13 @@ def test_fused_step_trajectories(sgdb, cuda_device, kind, dtype, P, pad):
     _trajectory(sgdb, cuda_device, 20, 16, P, 4, dtype, OPTS[kind], seed=41 + pad, pad=pad)
 
 
+@pytest.mark.parametrize("N,b", [(1, 0), (1, 5), (2, 1), (3, 0)])
+def test_few_kept_gradients(sgdb, cuda_device, N, b):
+    """N = 1 returns the single earliest current gradient; odd and even N take different branches of the row loop."""
+    _trajectory(sgdb, cuda_device, N + b, N, 20_011, 3, "f32", OPTS["momentum"], seed=43 + N + b)
+    _trajectory(sgdb, cuda_device, N + b, N, 20_011, 2, "bf16", OPTS["sgd"], seed=44 + N + b, pad=5)
+
+
 def test_config1_shape_reduced_columns(sgdb, cuda_device):
     """W=100, N=96, RMSProp with the Inception hyper-parameters, T=10, on a 1/100 column slice."""
     c = wl.CONFIGS[1]
@@ -358,7 +365,7 @@ def test_run_to_run_bitwise_determinism_and_tuning_independence(sgdb, cuda_devic
     arrival, tags = step_inputs(seed, 0, W, N)
     outs = []
     try:
-        for stages, ctas in ((0, 0), (0, 0), (3, 1), (20, 1), (5, 3)):
+        for stages, ctas in ((0, 0), (0, 0), (2, 1), (3, 1), (20, 1), (5, 3), (64, 8)):
             sgdb.sgdb_set_tuning(stages, ctas)
             theta = wl.theta0(seed, P, dev)
             s0, s1 = gpu_state("adam", P, dev)
