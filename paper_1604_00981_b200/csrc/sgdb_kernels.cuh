@@ -131,7 +131,8 @@ struct StreamParams {
   int stages;                   // ring depth
   const int32_t* order;         // [N] row ids in summation order (when the selection is given)
   const int32_t* info;          // optional [2]; info[1] != SGDB_OK: do nothing
-  int32_t* status_out;          // optional: receives SGDB_ERR_TIMEOUT if a wait runs out
+  int32_t* status_out;          // optional: receives SGDB_ERR_TIMEOUT if a wait runs out, or
+                                // SGDB_ERR_INVALID_ARG for an incomplete segment table entry
   // When `arrival` is not null the kernel takes the selection itself: every block
   // ranks the W workers in its prologue (the same deterministic result in each) and
   // block 0 writes mask_out, order_out and info_out.
@@ -253,12 +254,19 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
   }
   if (p.table != nullptr) {
     // tiles per segment, then an inclusive scan: prefix_s[i] = tiles in segments < i
+    // The same pass looks for entries that lack a pointer this rule needs (the host cannot
+    // see the table); their tiles are skipped below and block 0 reports them once.
+    int incomplete = 0;
     for (int i = tid; i < p.S; i += NT + 32) {
-      const long long len = p.table[i].len;
-      prefix_s[i + 1] = len > 0 ? static_cast<int>((len + TILE - 1) / TILE) : 0;
+      const sgdb_segment_t seg = p.table[i];
+      prefix_s[i + 1] = seg.len > 0 ? static_cast<int>((seg.len + TILE - 1) / TILE) : 0;
+      if (seg.len > 0 && (seg.theta == nullptr || seg.grad == nullptr || (Rule::kState0 && seg.state0 == nullptr) ||
+                          (Rule::kState1 && seg.state1 == nullptr)))
+        incomplete = 1;
     }
     if (tid == 0) prefix_s[0] = 0;
-    __syncthreads();
+    incomplete = __syncthreads_or(incomplete);
+    if (incomplete && blockIdx.x == 0 && tid == 0 && p.status_out != nullptr) *p.status_out = SGDB_ERR_INVALID_ARG;
     if (tid < 32) {
       int carry = 0;
       for (int base = 1; base <= p.S; base += 32) {
@@ -338,10 +346,7 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
       };
       const bool has_tail = td.bulk_cols < td.ncols;
 
-      if (td.bad) {
-        if (tid == 0 && p.status_out != nullptr) *p.status_out = SGDB_ERR_INVALID_ARG;
-        continue;
-      }
+      if (td.bad) continue;  // reported by block 0 in the prologue
       if (td.bulk_cols == 0) {
         for (int k = 0; k < N; ++k) add_row_tail(k);
       } else {
