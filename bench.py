@@ -244,6 +244,21 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None):
         torch.cuda.synchronize()
         return {"cuda_graph_replay_us_per_step": 1e3 * start.elapsed_time(stop) / (20 * N_SETS)}
 
+    def separate_calls():
+        """The same step as three calls (select, aggregate into a mean vector, update from it)."""
+        mean = torch.empty(P, device=dev)
+
+        def separate_step(i):
+            opt.step = i + 1
+            sgdb.sgdb_select(arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, mask, order, info)
+            sgdb.sgdb_aggregate(grad, P, N, order, info, mean)
+            sgdb.sgdb_update(theta, s0, s1, mean, opt, info)
+
+        ms = time_steps(separate_step, 10, 3)
+        moved = grad_bytes + 2 * (1 + n_state) * P * 4 + 2 * P * 4  # the mean is written and read back
+        return {"separate_calls_ms_per_step": ms, "separate_calls_total_gbs": moved / (ms * 1e-3) / 1e9,
+                "separate_calls_launches_per_step": 3}
+
     grad_bytes = int(kept_mean * P * grad.element_size())
     state = dict(grad=grad, theta=theta, s0=s0, s1=s1, opt=opt)
     total = grad_bytes + 2 * (1 + n_state) * P * 4 + (2 * P * 4 if ema else 0)
@@ -252,7 +267,7 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None):
                 % (cfg.grad_dtype, cfg.opt["kind"], " + parameter average" if ema else ""), state=state,
                 extra={"parameter_average": True} if ema else
                 ({"deadline_s": deadline, "mean_rows_kept": kept_mean} if deadline is not None else
-                 (graph_replay if P * W <= 1_000_000 else {})))
+                 (graph_replay if P * W <= 1_000_000 else separate_calls)))
 
 
 def setup_segmented(cfg, dev, sgdb, seed):
