@@ -69,9 +69,15 @@ class Opt:
 
 def _load():
     if not os.path.exists(LIB_PATH):
-        raise ImportError(
-            "libsgdb.so is not built (%s). Run `python -m paper_1604_00981_b200.build`; "
-            "this package has no CPU fallback." % LIB_PATH)
+        # not built yet: compile it now if the CUDA toolkit is here; there is nothing else to fall back to
+        try:
+            from . import build as _build
+
+            _build.build()
+        except Exception as e:
+            raise ImportError(
+                "libsgdb.so is not built (%s) and building it failed: %s. Run `python -m paper_1604_00981_b200.build`; "
+                "this package has no CPU fallback." % (LIB_PATH, e))
     lib = ctypes.CDLL(LIB_PATH)
     vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
     sigs = {
