@@ -24,7 +24,7 @@ _LIB = os.path.join(_HERE, "libsgdb_oracle.so")
 
 OK, INVALID, INSUFFICIENT = 0, 1, 2
 F32, BF16 = 0, 1
-SGD, MOMENTUM, RMSPROP, ADAM = 0, 1, 2, 3
+SGD, MOMENTUM, RMSPROP, ADAM, ADAGRAD = 0, 1, 2, 3, 4
 
 
 def build(force: bool = False) -> str:

@@ -36,7 +36,7 @@
 
 enum { ORACLE_OK = 0, ORACLE_INVALID = 1, ORACLE_INSUFFICIENT = 2 };
 enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
-enum { ORACLE_SGD = 0, ORACLE_MOMENTUM = 1, ORACLE_RMSPROP = 2, ORACLE_ADAM = 3 };
+enum { ORACLE_SGD = 0, ORACLE_MOMENTUM = 1, ORACLE_RMSPROP = 2, ORACLE_ADAM = 3, ORACLE_ADAGRAD = 4 };
 
 typedef struct {
   int32_t kind;
@@ -170,7 +170,9 @@ int oracle_aggregate(const void *grad, int dtype, int64_t P, int64_t ld, int32_t
  *             (Appendix A: "RMSProp with momentum", decay rho, momentum mu)
  *   Adam      m <- b1*m + (1-b1)*g;  v <- b2*v + (1-b2)*g^2;
  *             theta <- theta - lr * (m/(1-b1^k)) / (sqrt(v/(1-b2^k)) + eps),  k = step
- * s0/s1 hold (v,-), (s,m), (m,v) for momentum, RMSProp, Adam.
+ *   AdaGrad   s <- s + g^2;  theta <- theta - lr * g / (sqrt(s) + eps)
+ *             (named in the Introduction next to RMSProp and Adam; Duchi et al.'s rule)
+ * s0/s1 hold (v,-), (s,m), (m,v), (s,-) for momentum, RMSProp, Adam, AdaGrad.
  */
 int oracle_update(double *theta, double *s0, double *s1, const double *mean, int64_t P,
                   const oracle_opt_t *opt) {
@@ -197,6 +199,10 @@ int oracle_update(double *theta, double *s0, double *s1, const double *mean, int
         theta[i] = theta[i] - opt->lr * m_hat / (sqrt(v_hat) + opt->eps);
         break;
       }
+      case ORACLE_ADAGRAD:
+        s0[i] = s0[i] + g * g;
+        theta[i] = theta[i] - opt->lr * g / (sqrt(s0[i]) + opt->eps);
+        break;
       default:
         return ORACLE_INVALID;
     }

@@ -34,6 +34,8 @@ MUTANTS = [
     ("adam_no_bias_correction", "double m_hat = s0[i] / (1.0 - pow(opt->beta1, (double)opt->step));", "double m_hat = s0[i];"),
     ("adam_eps_inside", "(sqrt(v_hat) + opt->eps)", "sqrt(v_hat + opt->eps)"),
     ("adam_moments_swapped", "s1[i] = opt->beta2 * s1[i] + (1.0 - opt->beta2) * g * g;", "s1[i] = opt->beta1 * s1[i] + (1.0 - opt->beta1) * g * g;"),
+    ("adagrad_decays", "s0[i] = s0[i] + g * g;", "s0[i] = 0.9 * s0[i] + g * g;"),
+    ("adagrad_eps_inside", "theta[i] = theta[i] - opt->lr * g / (sqrt(s0[i]) + opt->eps);", "theta[i] = theta[i] - opt->lr * g / sqrt(s0[i] + opt->eps);"),
     ("ema_weights_swapped", "avg[i] = alpha * avg[i] + (1.0 - alpha) * theta[i];", "avg[i] = (1.0 - alpha) * avg[i] + alpha * theta[i];"),
     ("ema_of_updated_parameters", "if (rc == ORACLE_OK) oracle_ema(avg, theta_t, P, alpha);", "if (rc == ORACLE_OK) oracle_ema(avg, theta, P, alpha);"),
     ("ema_moves_without_update", "if (rc == ORACLE_OK) oracle_ema(avg, theta_t, P, alpha);", "oracle_ema(avg, theta_t, P, alpha);"),

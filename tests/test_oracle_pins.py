@@ -352,6 +352,22 @@ def test_rmsprop_learning_rate_enters_the_momentum_buffer():
     assert m.tolist() == [4.5, -4.5] and th.tolist() == [4.5, 15.5]
 
 
+def test_adagrad_closed_form():
+    """Constant g: s_k = k g^2, so with eps = 0 theta_k = theta_0 - lr sign(g) sum_{j<=k} 1/sqrt(j);
+    with eps > 0 each term is |g| / (sqrt(j) |g| + eps)."""
+    g = np.array([-3.0, -0.25, 0.5, 2.0])
+    traj = _run_constant(oracle.ADAGRAD, g, 7, lr=0.1, eps=0.0)
+    for k in range(1, 8):
+        np.testing.assert_allclose(traj[k - 1], 1.5 - 0.1 * np.sign(g) * sum(1 / math.sqrt(j) for j in range(1, k + 1)), rtol=1e-13)
+    traj = _run_constant(oracle.ADAGRAD, g, 5, lr=0.1, eps=0.5)
+    for k in range(1, 6):
+        step = sum(np.abs(g) / (math.sqrt(j) * np.abs(g) + 0.5) for j in range(1, k + 1))
+        np.testing.assert_allclose(traj[k - 1], 1.5 - 0.1 * np.sign(g) * step, rtol=1e-13)
+    th, acc = np.array([0.0]), np.array([5.0])  # the accumulator is the caller's: 5 + 2^2 = 9, root 3, eps 1 outside
+    oracle.update(th, acc, None, np.array([2.0]), oracle.Opt(kind=oracle.ADAGRAD, lr=1.0, eps=1.0))
+    assert acc[0] == 9.0 and th[0] == -0.5
+
+
 def test_adam_closed_form_every_step():
     lr, eps, k = 1e-3, 1e-8, 9
     traj = _run_constant(oracle.ADAM, G_CONST, k, lr=lr, beta1=0.9, beta2=0.999, eps=eps)
