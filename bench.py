@@ -136,7 +136,8 @@ def oracle_sample_run(cfg, P_sample: int, steps: int, warmup: int, seed_shift: i
     theta = wl.theta0(cfg.seed, P_sample, "cpu").numpy().astype(np.float64)
     s0, s1 = np.zeros(P_sample), np.zeros(P_sample)
     hyper = {k: float(np.float32(v)) for k, v in cfg.opt.items() if k != "kind"}
-    kind = {"sgd": oracle.SGD, "momentum": oracle.MOMENTUM, "rmsprop": oracle.RMSPROP, "adam": oracle.ADAM}[cfg.opt["kind"]]
+    kind = {"sgd": oracle.SGD, "momentum": oracle.MOMENTUM, "rmsprop": oracle.RMSPROP, "adam": oracle.ADAM,
+            "adagrad": oracle.ADAGRAD}[cfg.opt["kind"]]
     times = []
     for t in range(warmup + steps):
         arrival, tags = wl.arrivals(cfg.seed, t, W), wl.tags(cfg.seed, t, W, N)
@@ -172,7 +173,7 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
-N_STATE = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2}
+N_STATE = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2, "adagrad": 1}
 N_SETS = 16  # arrival/tag draws rotate, so the kept set differs from step to step
 
 

@@ -68,8 +68,9 @@ typedef enum {
   SGDB_SGD = 0,      /* theta -= lr * g                                   (Section 1.1, SGD rule)      */
   SGDB_MOMENTUM = 1, /* v = momentum*v + g;  theta -= lr * v                                           */
   SGDB_RMSPROP = 2,  /* s = decay*s + (1-decay)*g^2;  m = momentum*m + lr*g/sqrt(s+eps);  theta -= m   */
-  SGDB_ADAM = 3      /* m = beta1*m + (1-beta1)*g;  v = beta2*v + (1-beta2)*g^2;
+  SGDB_ADAM = 3,     /* m = beta1*m + (1-beta1)*g;  v = beta2*v + (1-beta2)*g^2;
                         theta -= lr * (m/(1-beta1^step)) / (sqrt(v/(1-beta2^step)) + eps)             */
+  SGDB_ADAGRAD = 4   /* s = s + g^2;  theta -= lr * g / (sqrt(s) + eps)                               */
 } sgdb_opt_kind_t;
 
 /*
@@ -79,7 +80,7 @@ typedef enum {
  * family (Section 1.1) and uses RMSProp with momentum in its experiments
  * (Appendix A) without printing equations; the forms above are the ones this
  * library computes.  state0/state1 per rule: SGD none; MOMENTUM v/-; RMSPROP
- * s/m; ADAM m/v.  `step` is the 1-based count of updates including this one and
+ * s/m; ADAM m/v; ADAGRAD s/-.  `step` is the 1-based count of updates including this one and
  * matters to ADAM only.
  */
 typedef struct sgdb_opt {

@@ -17,10 +17,11 @@ LIB_PATH = os.path.join(_HERE, "libsgdb.so")
 
 SGDB_OK, SGDB_ERR_INVALID_ARG, SGDB_ERR_INSUFFICIENT, SGDB_ERR_CUDA, SGDB_ERR_UNSUPPORTED, SGDB_ERR_TIMEOUT = range(6)
 SGDB_F32, SGDB_BF16 = 0, 1
-SGDB_SGD, SGDB_MOMENTUM, SGDB_RMSPROP, SGDB_ADAM = range(4)
+SGDB_SGD, SGDB_MOMENTUM, SGDB_RMSPROP, SGDB_ADAM, SGDB_ADAGRAD = range(5)
 SGDB_MAX_WORKERS = 1024
 SGDB_MAX_SEGMENTS = 4096
-_KINDS = {"sgd": SGDB_SGD, "momentum": SGDB_MOMENTUM, "rmsprop": SGDB_RMSPROP, "adam": SGDB_ADAM}
+_KINDS = {"sgd": SGDB_SGD, "momentum": SGDB_MOMENTUM, "rmsprop": SGDB_RMSPROP, "adam": SGDB_ADAM,
+          "adagrad": SGDB_ADAGRAD}
 
 EXPORTS = (
     "sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented",
@@ -51,7 +52,7 @@ class CSegment(ctypes.Structure):
 
 @dataclass
 class Opt:
-    """sgdb_opt_t.  `kind` is "sgd" | "momentum" | "rmsprop" | "adam" (or the enum value)."""
+    """sgdb_opt_t.  `kind` is "sgd" | "momentum" | "rmsprop" | "adam" | "adagrad" (or the enum value)."""
 
     kind: object = "sgd"
     lr: float = 0.1

@@ -127,6 +127,11 @@ sgdb_status_t prepare_rule(const sgdb_opt_t* opt, const void* state0, const void
       *ep = EP_ADAM;
       return SGDB_OK;
     }
+    case SGDB_ADAGRAD:
+      if (!std::isfinite(opt->eps) || state0 == nullptr) return SGDB_ERR_INVALID_ARG;
+      h->eps = opt->eps;
+      *ep = EP_ADAGRAD;
+      return SGDB_OK;
     default:
       return SGDB_ERR_INVALID_ARG;
   }
@@ -190,6 +195,7 @@ sgdb_status_t launch_stream_ep(int ep, const StreamParams& p, long long tiles, c
     case EP_MOMENTUM: return launch_stream_t<GT, EP_MOMENTUM>(p, tiles, stream);
     case EP_RMSPROP: return launch_stream_t<GT, EP_RMSPROP>(p, tiles, stream);
     case EP_ADAM: return launch_stream_t<GT, EP_ADAM>(p, tiles, stream);
+    case EP_ADAGRAD: return launch_stream_t<GT, EP_ADAGRAD>(p, tiles, stream);
   }
   return SGDB_ERR_INVALID_ARG;
 }
@@ -303,6 +309,7 @@ sgdb_status_t sgdb_update(float* d_theta, float* d_state0, float* d_state1, cons
     case EP_MOMENTUM: update_kernel<EP_MOMENTUM><<<static_cast<unsigned>(grid), 256, 0, s>>>(p); break;
     case EP_RMSPROP: update_kernel<EP_RMSPROP><<<static_cast<unsigned>(grid), 256, 0, s>>>(p); break;
     case EP_ADAM: update_kernel<EP_ADAM><<<static_cast<unsigned>(grid), 256, 0, s>>>(p); break;
+    case EP_ADAGRAD: update_kernel<EP_ADAGRAD><<<static_cast<unsigned>(grid), 256, 0, s>>>(p); break;
     default: return SGDB_ERR_INVALID_ARG;
   }
   return launch_status();
@@ -481,6 +488,7 @@ sgdb_status_t sgdb_accumulate_arrival(const void* d_row, sgdb_dtype_t dt, int32_
     SGDB_ARRIVAL_CASE(EP_MOMENTUM)
     SGDB_ARRIVAL_CASE(EP_RMSPROP)
     SGDB_ARRIVAL_CASE(EP_ADAM)
+    SGDB_ARRIVAL_CASE(EP_ADAGRAD)
     default: return SGDB_ERR_INVALID_ARG;
   }
 #undef SGDB_ARRIVAL_CASE

@@ -10,7 +10,7 @@
 namespace sgdb {
 
 // Epilogue selector of the row-streaming kernel: write the mean, or apply a rule.
-enum : int { EP_MEAN = 0, EP_SGD = 1, EP_MOMENTUM = 2, EP_RMSPROP = 3, EP_ADAM = 4 };
+enum : int { EP_MEAN = 0, EP_SGD = 1, EP_MOMENTUM = 2, EP_RMSPROP = 3, EP_ADAM = 4, EP_ADAGRAD = 5 };
 
 // Hyper-parameters as the kernels use them; derived once on the host.
 struct Hyper {
@@ -208,6 +208,9 @@ __device__ __forceinline__ void apply_rule(const Hyper& h, float g, float& theta
     float m_hat = __fdiv_rn(s0, h.bc1);
     float v_hat = __fdiv_rn(s1, h.bc2);
     theta = __fsub_rn(theta, __fdiv_rn(__fmul_rn(h.lr, m_hat), __fadd_rn(__fsqrt_rn(v_hat), h.eps)));
+  } else if (EP == EP_ADAGRAD) {
+    s0 = __fmaf_rn(g, g, s0);
+    theta = __fsub_rn(theta, __fdiv_rn(__fmul_rn(h.lr, g), __fadd_rn(__fsqrt_rn(s0), h.eps)));
   }
 }
 
@@ -219,7 +222,7 @@ __device__ __forceinline__ float ema_rule(float alpha, float one_minus_alpha, fl
 template <int EP>
 struct RuleTraits {
   static constexpr bool kTheta = EP != EP_MEAN;
-  static constexpr bool kState0 = EP == EP_MOMENTUM || EP == EP_RMSPROP || EP == EP_ADAM;
+  static constexpr bool kState0 = EP == EP_MOMENTUM || EP == EP_RMSPROP || EP == EP_ADAM || EP == EP_ADAGRAD;
   static constexpr bool kState1 = EP == EP_RMSPROP || EP == EP_ADAM;
 };
 

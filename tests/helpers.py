@@ -16,10 +16,12 @@ OPTS = {
     "momentum": dict(kind="momentum", lr=0.01, momentum=0.9),
     "rmsprop": dict(kind="rmsprop", lr=0.045, decay=0.9, momentum=0.9, eps=1.0),
     "adam": dict(kind="adam", lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8),
+    "adagrad": dict(kind="adagrad", lr=0.05, eps=1e-7),
 }
 
-_ORACLE_KIND = {"sgd": oracle.SGD, "momentum": oracle.MOMENTUM, "rmsprop": oracle.RMSPROP, "adam": oracle.ADAM}
-STATES = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2}
+_ORACLE_KIND = {"sgd": oracle.SGD, "momentum": oracle.MOMENTUM, "rmsprop": oracle.RMSPROP, "adam": oracle.ADAM,
+                "adagrad": oracle.ADAGRAD}
+STATES = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2, "adagrad": 1}
 
 
 def rel_err(x, y) -> float:

@@ -46,7 +46,7 @@ def _make_model(dev, lengths, W, kind, dtype, seed, packed):
             s0, s1 = torch.zeros(L, device=dev), torch.zeros(L, device=dev)
             ld = (L + vec - 1) // vec * vec
             grad = wl.grad_matrix(seed + i, 0, W, L, scales, dtype, dev, ld=ld, pad_value=float("nan"))
-        n = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2}[kind]
+        n = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2, "adagrad": 1}[kind]
         segs.append((theta, s0 if n >= 1 else None, s1 if n >= 2 else None, grad))
         off += L
     return segs, scales
@@ -64,7 +64,8 @@ def _regen(segs, scales, seed, t, W, dtype, dev, packed):
 
 
 @pytest.mark.parametrize("packed", [False, True])
-@pytest.mark.parametrize("kind,dtype", [("momentum", "f32"), ("adam", "bf16"), ("sgd", "f32"), ("rmsprop", "bf16")])
+@pytest.mark.parametrize("kind,dtype", [("momentum", "f32"), ("adam", "bf16"), ("sgd", "f32"), ("rmsprop", "bf16"),
+                                        ("adagrad", "f32")])
 def test_segmented_step_matches_oracle_and_per_tensor_launches(sgdb, cuda_device, kind, dtype, packed):
     dev = cuda_device
     W, N, T, seed = 14, 11, 3, 101
@@ -159,7 +160,7 @@ def test_segmented_edge_cases(sgdb, cuda_device):
 @pytest.mark.parametrize("kind,dtype,P,b", [("rmsprop", "f32", 100_003, 0), ("rmsprop", "f32", 100_003, 2),
                                             ("rmsprop", "f32", 65_536, 4), ("rmsprop", "f32", 100_003, 8),
                                             ("adam", "bf16", 50_001, 3), ("sgd", "f32", 5, 1),
-                                            ("momentum", "bf16", 4099, 2)])
+                                            ("momentum", "bf16", 4099, 2), ("adagrad", "f32", 30_001, 2)])
 def test_accumulate_on_arrival(sgdb, cuda_device, kind, dtype, P, b):
     """Rows are delivered one per call in arrival sequence, stale rows and late rows included.  Outcomes
     and counts match the oracle's replay of Algorithm 4; parameters match the oracle within tolerance
