@@ -43,7 +43,7 @@ NOMINAL_HBM_GBS = 8000.0
 
 # DRAM traffic of one fused-step launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
 # as bytes per algorithmic byte; valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"src_digest": "6382a9247a2cbd49", "dram_bytes_per_algorithmic_byte": 0.9952}
+NCU_TRAFFIC = {"src_digest": "aafc1221a3f99157", "dram_bytes_per_algorithmic_byte": 0.9948}
 
 
 def kernel_source_digest() -> str:
