@@ -71,11 +71,11 @@ def _flat_trajectory_sampled(sgdb, dev, cfg, T):
 
 
 def test_config1_full_size(sgdb, cuda_device):
-    """P = 23.8 M fp32, W = 100 (N = 96, b = 4), RMSProp; fused step vs oracle at sampled columns, then the
+    """P = 23.8 M fp32, W = 100 (N = 96, b = 4), RMSProp, T = 10 steps; fused step vs oracle at sampled columns, then the
     separate select / aggregate / update calls against the fused step on the whole vector."""
     _need_memory(cuda_device, 12)
     dev, cfg = cuda_device, wl.CONFIGS[1]
-    grad, theta, s0, s1, arrival, tags, t = _flat_trajectory_sampled(sgdb, dev, cfg, T=3)
+    grad, theta, s0, s1, arrival, tags, t = _flat_trajectory_sampled(sgdb, dev, cfg, T=cfg.T)
     W, N, P = cfg.W, cfg.N, cfg.P
     th_f, s0_f, s1_f = theta.clone(), s0.clone(), s1.clone()
     mask, order, info = selection_buffers(W, N, dev)
@@ -92,9 +92,9 @@ def test_config1_full_size(sgdb, cuda_device):
 
 
 def test_config3_full_size(sgdb, cuda_device):
-    """P = 100 M, W = 208 (N = 200, b = 8), bf16 rows (41.6 GB), Adam."""
+    """P = 100 M, W = 208 (N = 200, b = 8), bf16 rows (41.6 GB), Adam, T = 5 steps."""
     _need_memory(cuda_device, 48)
-    _flat_trajectory_sampled(sgdb, cuda_device, wl.CONFIGS[3], T=2)
+    _flat_trajectory_sampled(sgdb, cuda_device, wl.CONFIGS[3], T=wl.CONFIGS[3].T)
 
 
 def test_config2_full_size_segmented(sgdb, cuda_device):
