@@ -37,6 +37,37 @@ def test_binding_exposes_the_same_names():
     assert set(binding.EXPORTS) == set(_declared())
 
 
+def test_header_is_plain_c_and_links_from_c(tmp_path, lib):
+    """The boundary is a C ABI: the header compiles as C11 with gcc, and a C program linked against the
+    library can call it (host-checked error paths only, so no GPU is needed)."""
+    import subprocess
+    from paper_1604_00981_b200 import build
+
+    src = tmp_path / "use_sgdb.c"
+    src.write_text("""
+#include <stdio.h>
+#include "sgdb.h"
+int main(void) {
+  sgdb_opt_t opt = {SGDB_RMSPROP, 0.045f, 0.9f, 0.9f, 0.f, 0.f, 1.0f, 1};
+  sgdb_segment_t seg = {0, 0, 0, 0, 0, 0};
+  (void)seg;
+  if (sgdb_select(0, 0, 0, 1, 0, 0, 0, 0, 0) != SGDB_ERR_INVALID_ARG) return 1;
+  if (sgdb_update(0, 0, 0, 0, 4, &opt, 0, 0) != SGDB_ERR_INVALID_ARG) return 2;
+  if (sgdb_step_host_workspace_bytes(SGDB_F32, 10, 10, 5, 1) < 240) return 3;
+  if (sgdb_learning_rate(2.0, 0.25, 1, 1, 1.0) != 1.0) return 4;
+  printf("%d %s\\n", sgdb_version(), sgdb_strerror(SGDB_ERR_INSUFFICIENT));
+  return 0;
+}
+""")
+    exe = tmp_path / "use_sgdb"
+    libdir = os.path.dirname(build.LIB)
+    subprocess.run(["gcc", "-std=c11", "-Wall", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"), str(src),
+                    "-o", str(exe), "-L", libdir, "-lsgdb", "-Wl,-rpath," + libdir, "-lm"], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, (out.returncode, out.stderr)
+    assert out.stdout.split()[0] == str(lib.sgdb_version())
+
+
 def test_version_and_strerror(lib):
     lib.sgdb_strerror.restype = ctypes.c_char_p
     assert lib.sgdb_version() >= 100
