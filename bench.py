@@ -43,15 +43,20 @@ NOMINAL_HBM_GBS = 8000.0
 
 # DRAM traffic of one fused-step launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
 # as bytes per algorithmic byte; valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"src_digest": "aafc1221a3f99157", "dram_bytes_per_algorithmic_byte": 0.9948}
+NCU_TRAFFIC = {"src_digest": "f559b579ce14cf57", "dram_bytes_per_algorithmic_byte": 0.9948}
 
 
 def kernel_source_digest() -> str:
+    """Digest of the device code the fused step runs: the shared device header, and the kernel file up to
+    the end of the row-streaming kernel (selection prologue included)."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_1604_00981_b200", "csrc")
-    for name in sorted(n for n in os.listdir(csrc) if n.endswith(".cuh")):  # device code only
-        with open(os.path.join(csrc, name), "rb") as f:
-            h.update(f.read())
+    with open(os.path.join(csrc, "sgdb_device.cuh"), "rb") as f:
+        h.update(f.read())
+    with open(os.path.join(csrc, "sgdb_kernels.cuh"), "rb") as f:
+        text = f.read()
+    end = text.find(b"// ====================================================================== update from a mean")
+    h.update(text if end < 0 else text[:end])
     return h.hexdigest()[:16]
 
 
