@@ -84,6 +84,7 @@ def _load():
             "oracle_step",
             "oracle_accumulate_arrival",
             "oracle_step_ema",
+            "oracle_accumulate_arrival_ema",
             "oracle_select_deadline",
             "oracle_step_deadline",
         ):
@@ -255,6 +256,22 @@ def accumulate_arrival(row, row_tag: int, t: int, N: int, acc, state, theta, s0,
         _p(r), ctypes.c_int(dt), ctypes.c_int32(row_tag), ctypes.c_int32(t), ctypes.c_int32(N),
         ctypes.c_int64(P), _p(acc), _p(state), _p(theta), _p(s0), _p(s1), ctypes.byref(c),
         ctypes.byref(outcome),
+    )
+    assert rc == OK, rc
+    return outcome.value
+
+
+def accumulate_arrival_ema(row, row_tag: int, t: int, N: int, acc, state, theta, s0, s1, opt: Opt, avg, alpha: float) -> int:
+    """accumulate_arrival plus the parameter average, which moves only when the N-th gradient fires the update."""
+    r, dt = _grad(row)
+    P = len(theta)
+    assert acc.dtype == np.float64 and state.dtype == np.int32 and len(state) == 3 and avg.dtype == np.float64
+    outcome = ctypes.c_int32(-1)
+    c = opt._c()
+    rc = _load().oracle_accumulate_arrival_ema(
+        _p(r), ctypes.c_int(dt), ctypes.c_int32(row_tag), ctypes.c_int32(t), ctypes.c_int32(N),
+        ctypes.c_int64(P), _p(acc), _p(state), _p(theta), _p(s0), _p(s1), ctypes.byref(c), _p(avg),
+        ctypes.c_double(alpha), ctypes.byref(outcome),
     )
     assert rc == OK, rc
     return outcome.value

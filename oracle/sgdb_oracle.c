@@ -282,6 +282,24 @@ double oracle_learning_rate(double gamma0, double beta, int64_t t, int64_t N, do
  */
 int oracle_accumulate_arrival(const void *row, int dtype, int32_t row_tag, int32_t t, int32_t N,
                               int64_t P, double *acc, int32_t *state, double *theta, double *s0,
+                              double *s1, const oracle_opt_t *opt, int32_t *outcome);
+
+/* The same with Algorithm 4's last line: when the N-th gradient triggers the update, the average takes in
+ * the parameters as they were before it (avg may be NULL: no average is kept). */
+int oracle_accumulate_arrival_ema(const void *row, int dtype, int32_t row_tag, int32_t t, int32_t N,
+                                  int64_t P, double *acc, int32_t *state, double *theta, double *s0,
+                                  double *s1, const oracle_opt_t *opt, double *avg, double alpha,
+                                  int32_t *outcome) {
+  double *theta_t = (double *)malloc(sizeof(double) * (size_t)(P > 0 ? P : 1));
+  memcpy(theta_t, theta, sizeof(double) * (size_t)P);
+  int rc = oracle_accumulate_arrival(row, dtype, row_tag, t, N, P, acc, state, theta, s0, s1, opt, outcome);
+  if (rc == ORACLE_OK && *outcome == 2 && avg != NULL) oracle_ema(avg, theta_t, P, alpha);
+  free(theta_t);
+  return rc;
+}
+
+int oracle_accumulate_arrival(const void *row, int dtype, int32_t row_tag, int32_t t, int32_t N,
+                              int64_t P, double *acc, int32_t *state, double *theta, double *s0,
                               double *s1, const oracle_opt_t *opt, int32_t *outcome) {
   if (N < 1 || P < 0) return ORACLE_INVALID;
   state[1] += 1;

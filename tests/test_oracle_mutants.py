@@ -45,6 +45,10 @@ MUTANTS = [
     ("deadline_ignored", "if (!(arrival[w] <= deadline)) continue;", ""),
     ("deadline_drops_last_kept", "rc = oracle_aggregate(grad, dtype, P, ld, *n_kept, order, mean); /* divisor: the number kept */",
      "rc = oracle_aggregate(grad, dtype, P, ld, (*n_kept > 1 ? *n_kept - 1 : 1), order, mean);"),
+    ("arrival_average_moves_every_time", "if (rc == ORACLE_OK && *outcome == 2 && avg != NULL) oracle_ema(avg, theta_t, P, alpha);",
+     "if (rc == ORACLE_OK && *outcome >= 1 && avg != NULL) oracle_ema(avg, theta_t, P, alpha);"),
+    ("arrival_average_of_updated", "if (rc == ORACLE_OK && *outcome == 2 && avg != NULL) oracle_ema(avg, theta_t, P, alpha);",
+     "if (rc == ORACLE_OK && *outcome == 2 && avg != NULL) oracle_ema(avg, theta, P, alpha);"),
     ("arrival_counts_stale", "if (row_tag != t || t < state[2] || state[0] >= N) {", "if (t < state[2] || state[0] >= N) {"),
     ("arrival_never_closes", "state[2] = t + 1;", "state[2] = state[2];"),
     ("arrival_divides_late", "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)N;", "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)(N + 1);"),
@@ -76,7 +80,7 @@ def test_mutant_is_caught_by_a_pin(tmp_path, name, old, new):
                    check=True)
     lib = ctypes.CDLL(str(so_path))
     for fn_name in ("oracle_select", "oracle_aggregate", "oracle_update", "oracle_step", "oracle_accumulate_arrival",
-                    "oracle_step_ema", "oracle_select_deadline", "oracle_step_deadline"):
+                    "oracle_step_ema", "oracle_select_deadline", "oracle_step_deadline", "oracle_accumulate_arrival_ema"):
         getattr(lib, fn_name).restype = ctypes.c_int
     lib.oracle_ema.restype = None
     lib.oracle_learning_rate.restype = ctypes.c_double

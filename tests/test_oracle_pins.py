@@ -554,3 +554,26 @@ def test_arrival_server_with_n_equal_one_is_algorithm2():
         out = oracle.accumulate_arrival(rows[k], k, k, 1, acc, state, theta, None, None, oracle.Opt(kind=oracle.SGD, lr=lr))
         assert out == 2 and state.tolist() == [0, k + 1, k + 1]
     np.testing.assert_allclose(theta, theta0 - lr * rows.astype(np.float64).sum(axis=0), rtol=0, atol=1e-13)
+
+
+def test_arrival_server_with_average_equals_batched_step_with_average():
+    rng = np.random.default_rng(41)
+    W, N, P, T, alpha = 7, 5, 60, 4, 0.8
+    th_a = rng.normal(size=P)
+    th_b, avg_a, avg_b = th_a.copy(), th_a.copy(), th_a.copy()
+    acc, state = np.zeros(P), oracle.new_server_state()
+    for t in range(T):
+        grad = rng.normal(size=(W, P)).astype(np.float32)
+        arrival = rng.lognormal(0, 0.3, W).astype(np.float32)
+        tags = np.full(W, t, np.int32)
+        tags[int(rng.integers(0, W))] = t - 1
+        opt = oracle.Opt(kind=oracle.SGD, lr=0.1)
+        rc, *_ = oracle.step_ema(grad, P, arrival, tags, t, N, W - N, th_b, None, None, opt, avg_b, alpha)
+        assert rc == oracle.OK
+        before = avg_a.copy()
+        for i, w in enumerate(np.argsort(arrival, kind="stable")):
+            out = oracle.accumulate_arrival_ema(grad[w], int(tags[w]), t, N, acc, state, th_a, None, None, opt, avg_a, alpha)
+            if out != 2 and state[2] == t:
+                assert (avg_a == before).all()  # the average only moves when the update fires
+        np.testing.assert_allclose(th_a, th_b, rtol=1e-13, atol=1e-14)
+        np.testing.assert_allclose(avg_a, avg_b, rtol=1e-13, atol=1e-14)
