@@ -264,6 +264,17 @@ sgdb_status_t sgdb_accumulate_arrival(const void *d_row, sgdb_dtype_t dt, int32_
                                       void *stream);
 
 /*
+ * sgdb_accumulate_arrival_ema -- sgdb_accumulate_arrival that also keeps the parameter
+ * average of Algorithm 4's last line: d_ema [P] (fp32, 16-byte aligned) is updated as in
+ * sgdb_step_ema, in the launch of the N-th accepted gradient and only then.
+ */
+sgdb_status_t sgdb_accumulate_arrival_ema(const void *d_row, sgdb_dtype_t dt, int32_t row_tag,
+                                          int32_t t, int32_t N, int64_t P, float *d_acc,
+                                          int32_t *d_counter, float *d_theta, float *d_state0,
+                                          float *d_state1, const sgdb_opt_t *opt, float *d_ema,
+                                          float alpha, int32_t *d_info, void *stream);
+
+/*
  * sgdb_step_host -- sgdb_step for a server whose gradients arrive in HOST memory
  * (the worker-to-server message of Algorithm 3 lands in host buffers) and whose
  * new parameters go back out to the workers (Algorithm 3 reads theta each

@@ -25,7 +25,7 @@ _KINDS = {"sgd": SGDB_SGD, "momentum": SGDB_MOMENTUM, "rmsprop": SGDB_RMSPROP, "
 
 EXPORTS = (
     "sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented",
-    "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
+    "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_accumulate_arrival_ema", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
     "sgdb_set_tuning", "sgdb_strerror", "sgdb_version",
 )
 SGDB_STATIC_SCRATCH_BYTES = 8 << 20
@@ -95,6 +95,8 @@ def _load():
         "sgdb_learning_rate": (ctypes.c_double, [ctypes.c_double, ctypes.c_double, i64, i64, ctypes.c_double]),
         "sgdb_step_segmented": (i32, [vp, i32, i32, vp, vp, i32, i32, i32, ctypes.POINTER(_COpt), vp, vp, vp, vp]),
         "sgdb_accumulate_arrival": (i32, [vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, ctypes.POINTER(_COpt), vp, vp]),
+        "sgdb_accumulate_arrival_ema": (i32, [vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, ctypes.POINTER(_COpt), vp,
+                                              ctypes.c_float, vp, vp]),
         "sgdb_step_host": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt),
                                  vp, vp, vp, vp, vp, sz, vp]),
         "sgdb_step_host_workspace_bytes": (sz, [i32, i64, i64, i32, i32]),
@@ -286,6 +288,19 @@ def sgdb_accumulate_arrival(row, row_tag: int, t: int, N: int, acc, counter, the
                                         _dev(state1, torch.float32, "state1"), ctypes.byref(c),
                                         _dev(info, torch.int32, "info"), _stream(stream)),
            "sgdb_accumulate_arrival")
+
+
+def sgdb_accumulate_arrival_ema(row, row_tag: int, t: int, N: int, acc, counter, theta, state0, state1, opt: Opt, ema,
+                                alpha: float, info, P: int | None = None, stream=None) -> None:
+    """sgdb_accumulate_arrival that also moves the parameter average when the N-th gradient fires the update."""
+    P = theta.numel() if P is None else P
+    c = opt._c()
+    _check(_lib.sgdb_accumulate_arrival_ema(_dev(row, None, "row"), _grad_dtype(row), row_tag, t, N, P,
+                                            _dev(acc, torch.float32, "acc"), _dev(counter, torch.int32, "counter"),
+                                            _dev(theta, torch.float32, "theta"), _dev(state0, torch.float32, "state0"),
+                                            _dev(state1, torch.float32, "state1"), ctypes.byref(c),
+                                            _dev(ema, torch.float32, "ema"), alpha, _dev(info, torch.int32, "info"),
+                                            _stream(stream)), "sgdb_accumulate_arrival_ema")
 
 
 def sgdb_step_host_workspace_bytes(grad_dtype, P: int, ld: int, N: int, b: int) -> int:

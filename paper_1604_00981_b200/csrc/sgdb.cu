@@ -443,14 +443,14 @@ sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, s
   return launch_stream(dt, ep, p, 0, s);
 }
 
-sgdb_status_t sgdb_accumulate_arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag, int32_t t,
-                                      int32_t N, int64_t P, float* d_acc, int32_t* d_counter,
-                                      float* d_theta, float* d_state0, float* d_state1,
-                                      const sgdb_opt_t* opt, int32_t* d_info, void* stream) {
+static sgdb_status_t arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag, int32_t t, int32_t N, int64_t P,
+                             float* d_acc, int32_t* d_counter, float* d_theta, float* d_state0, float* d_state1,
+                             const sgdb_opt_t* opt, float* d_ema, float alpha, int32_t* d_info, void* stream) {
   if (d_row == nullptr || d_acc == nullptr || d_counter == nullptr || d_theta == nullptr || d_info == nullptr)
     return SGDB_ERR_INVALID_ARG;
   if (!dtype_ok(dt) || N < 1 || P < 0) return SGDB_ERR_INVALID_ARG;
-  if (!is_aligned16(d_acc) || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
+  if (!is_aligned16(d_acc) || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1) ||
+      !is_aligned16(d_ema))
     return SGDB_ERR_INVALID_ARG;
   Hyper h;
   int ep = 0;
@@ -459,7 +459,8 @@ sgdb_status_t sgdb_accumulate_arrival(const void* d_row, sgdb_dtype_t dt, int32_
   const DeviceInfo* dev = nullptr;
   st = device_info(&dev);
   if (st != SGDB_OK) return st;
-  ArrivalParams p{d_row, row_tag, t, N, P, d_acc, d_counter, d_theta, d_state0, d_state1, d_info, h};
+  ArrivalParams p{d_row, row_tag, t, N, P, d_acc, d_counter, d_theta, d_state0, d_state1, d_info,
+                  d_ema, alpha, static_cast<float>(1.0 - static_cast<double>(alpha)), h};
   const int V = dt == SGDB_BF16 ? 8 : 4;
   const long long chunks = (P + V - 1) / V;
   long long grid = (chunks + 4 * 256 - 1) / (4 * 256);  // 4 chunks per thread and pass
@@ -493,6 +494,24 @@ sgdb_status_t sgdb_accumulate_arrival(const void* d_row, sgdb_dtype_t dt, int32_
   }
 #undef SGDB_ARRIVAL_CASE
   return launch_status();
+}
+
+sgdb_status_t sgdb_accumulate_arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag, int32_t t,
+                                      int32_t N, int64_t P, float* d_acc, int32_t* d_counter,
+                                      float* d_theta, float* d_state0, float* d_state1,
+                                      const sgdb_opt_t* opt, int32_t* d_info, void* stream) {
+  return arrival(d_row, dt, row_tag, t, N, P, d_acc, d_counter, d_theta, d_state0, d_state1, opt, nullptr, 0.0f, d_info,
+                 stream);
+}
+
+sgdb_status_t sgdb_accumulate_arrival_ema(const void* d_row, sgdb_dtype_t dt, int32_t row_tag, int32_t t,
+                                          int32_t N, int64_t P, float* d_acc, int32_t* d_counter,
+                                          float* d_theta, float* d_state0, float* d_state1,
+                                          const sgdb_opt_t* opt, float* d_ema, float alpha, int32_t* d_info,
+                                          void* stream) {
+  if (d_ema == nullptr || !(alpha >= 0.0f && alpha <= 1.0f)) return SGDB_ERR_INVALID_ARG;
+  return arrival(d_row, dt, row_tag, t, N, P, d_acc, d_counter, d_theta, d_state0, d_state1, opt, d_ema, alpha, d_info,
+                 stream);
 }
 
 // Workspace layout of sgdb_step_host: arrival[W] f32 | tags[W] i32 | order[N] i32 | info[2] i32 |

@@ -568,6 +568,8 @@ struct ArrivalParams {
   float* s0;
   float* s1;
   int32_t* info;  // [2]
+  float* ema;     // optional: average of the parameters, moved when the update fires
+  float ema_alpha, ema_one_minus_alpha;
   Hyper h;
 };
 
@@ -663,6 +665,13 @@ __global__ void __launch_bounds__(256, 4) accumulate_arrival_kernel(const Arriva
         load_floats<V>(p.theta + i, vec, n, th);
         if (Rule::kState0) load_floats<V>(p.s0 + i, vec, n, s0);
         if (Rule::kState1) load_floats<V>(p.s1 + i, vec, n, s1);
+        if (p.ema != nullptr) {  // the average takes in theta as it is before this update
+          float avg[V];
+          load_floats<V>(p.ema + i, vec, n, avg);
+#pragma unroll
+          for (int e = 0; e < V; ++e) avg[e] = ema_rule(p.ema_alpha, p.ema_one_minus_alpha, avg[e], th[e]);
+          store_floats<V>(p.ema + i, vec, n, avg);
+        }
 #pragma unroll
         for (int e = 0; e < V; ++e) {
           a[e] = __fadd_rn(a[e], x[e]);

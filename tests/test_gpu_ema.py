@@ -55,6 +55,46 @@ def test_step_with_parameter_average(sgdb, cuda_device, kind, dtype, P, pad, alp
     assert torch.equal(theta, twin[0]) and torch.equal(avg, twin[1])  # fused == separate, bit for bit
 
 
+@pytest.mark.parametrize("kind,dtype", [("rmsprop", "f32"), ("adagrad", "bf16")])
+def test_arrival_mode_with_parameter_average(sgdb, cuda_device, kind, dtype):
+    """Row by row delivery: the average moves only in the launch that fires the update; results equal the fused
+    sgdb_step_ema bit for bit and the oracle within tolerance."""
+    dev = cuda_device
+    N, b, P, T, seed, alpha = 9, 2, 40_003, 3, 211, 0.9
+    W = N + b
+    scales = wl.worker_scales(seed, W)
+    theta = wl.theta0(seed, P, dev)
+    avg = theta.clone()
+    s0, s1 = gpu_state(kind, P, dev)
+    fused = (theta.clone(), avg.clone()) + gpu_state(kind, P, dev)
+    acc = torch.empty(P, device=dev)
+    counter = torch.zeros(4, dtype=torch.int32, device=dev)
+    info = torch.zeros(2, dtype=torch.int32, device=dev)
+    th_o = theta.cpu().numpy().astype(np.float64)
+    avg_o = th_o.copy()
+    s0_o, s1_o = oracle_state(kind, P)
+    acc_o, state_o = np.zeros(P), oracle.new_server_state()
+    mask, order, finfo = selection_buffers(W, N, dev)
+    for t in range(T):
+        grad = wl.grad_matrix(seed, t, W, P, scales, dtype, dev)
+        grad_h = wl.as_oracle_array(grad)
+        arrival, tags = step_inputs(seed, t, W, N)
+        for w in wl.delivery_sequence(arrival):
+            before = avg.clone()
+            sgdb.sgdb_accumulate_arrival_ema(grad[w], int(tags[w]), t, N, acc, counter, theta, s0, s1,
+                                             gpu_opt(OPTS[kind], t + 1), avg, alpha, info)
+            want = oracle.accumulate_arrival_ema(grad_h[w], int(tags[w]), t, N, acc_o, state_o, th_o, s0_o, s1_o,
+                                                 oracle_opt(OPTS[kind], t + 1), avg_o, f32(alpha))
+            assert info.cpu().tolist()[0] == want
+            if want != 2:
+                assert torch.equal(avg, before)  # the average waits for the update
+        sgdb.sgdb_step_ema(grad, P, to_dev(arrival, dev), to_dev(tags, dev), t, N, b, fused[0], fused[2], fused[3],
+                           gpu_opt(OPTS[kind], t + 1), fused[1], alpha, mask, order, finfo)
+        assert torch.equal(theta, fused[0]) and torch.equal(avg, fused[1])
+    tol = TOL_F32 if dtype == "f32" else TOL_BF16
+    assert rel_err(theta.cpu().numpy(), th_o) < tol and rel_err(avg.cpu().numpy(), avg_o) < tol
+
+
 def test_average_untouched_when_gradients_are_insufficient_and_bad_arguments(sgdb, cuda_device):
     dev = cuda_device
     W, N, P = 6, 5, 10_000
