@@ -4,21 +4,26 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl native|reference]
 
 A step is one pass of the whole path over one batch of synthetic input: select the first N of the
-N+b gradients, average them, apply RMSProp with momentum.  The workload is the Inception-v3-sized
-one: P = 23.8 M fp32 parameters, W = 100 (N = 96, b = 4).  Prints one JSON line.
+N+b gradients, average them, apply RMSProp with momentum.  The headline workload is the
+Inception-v3-sized one: P = 23.8 M fp32 parameters, W = 100 (N = 96, b = 4).  Prints one JSON line.
 
 value     gradient bytes read per second (N * P * 4 per step), inputs resident in HBM
 e2e       the same metric through sgdb_step_host: gradients, arrival times and tags start in pinned
           host memory, the updated parameters are read back, all inside the timed region
 roofline  algorithmic bytes of a step (gradient rows + parameters and state read and written) over
           the measured step time, against the measured HBM copy bandwidth of this machine
+extra     (one GPU, default workload) the spread of single-step times, a sustained run of at least
+          two seconds with the clocks seen, the same step as three separate calls, and the other
+          four seeded workloads: tiny SGD, 300-tensor segmented, bf16 rows + Adam, arrival by arrival
 With --gpus N > 1 (under torchrun) every rank is one parameter-server shard holding its own P
 columns; there is no data-path collective, and the value is the sum over ranks over the slowest rank.
---impl reference times the CPU oracle on a bounded column sample of the same workload.
+--impl reference times the CPU oracle on the same workload (all host cores, column ranges split
+over threads; the single-thread figure beside it).
 """
 from __future__ import annotations
 
 import argparse
+import gc
 import hashlib
 import json
 import os
@@ -73,7 +78,7 @@ class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw")
 
     def __init__(self, index: int):
         self.index = str(index)
@@ -110,7 +115,7 @@ class ClockSampler:
             self.thread.join(timeout=2)
 
     def summary(self):
-        sm, smax, reasons = [], [], set()
+        sm, smax, power, reasons = [], [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         for line in self.lines:
             parts = [p.strip() for p in line.split(",")]
@@ -124,59 +129,157 @@ class ClockSampler:
             for name, val in zip(names, parts[2:6]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
+            try:
+                power.append(float(parts[6]))
+            except (IndexError, ValueError):
+                pass
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
-                "samples": len(sm)}
+        out = {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+               "samples": len(sm)}
+        if power:
+            out["power_w_max"] = float(max(power))
+        return out
 
 
-def oracle_sample_run(cfg, P_sample: int, steps: int, warmup: int, seed_shift: int = 0):
-    """Times the CPU oracle, as it stands, on the first P_sample columns of the workload.
-    Returns (seconds per step, gradient GB/s)."""
+# ====================================================================== the CPU oracle as a baseline
+
+
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def host_cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def column_ranges(P: int, parts: int):
+    """[c0, c1) ranges that split P columns into `parts` nearly equal contiguous pieces (empty ones left out)."""
+    edges = [P * k // parts for k in range(parts + 1)]
+    return [(edges[k], edges[k + 1]) for k in range(parts) if edges[k + 1] > edges[k]]
+
+
+def _oracle_kind(cfg):
     import oracle
 
-    W, N = cfg.W, cfg.N
-    scales = wl.worker_scales(cfg.seed, W)
-    grad = wl.as_oracle_array(wl.grad_matrix(cfg.seed + seed_shift, 0, W, P_sample, scales, cfg.grad_dtype, "cpu"))
-    theta = wl.theta0(cfg.seed, P_sample, "cpu").numpy().astype(np.float64)
-    s0, s1 = np.zeros(P_sample), np.zeros(P_sample)
-    hyper = {k: float(np.float32(v)) for k, v in cfg.opt.items() if k != "kind"}
-    kind = {"sgd": oracle.SGD, "momentum": oracle.MOMENTUM, "rmsprop": oracle.RMSPROP, "adam": oracle.ADAM,
+    return {"sgd": oracle.SGD, "momentum": oracle.MOMENTUM, "rmsprop": oracle.RMSPROP, "adam": oracle.ADAM,
             "adagrad": oracle.ADAGRAD}[cfg.opt["kind"]]
+
+
+def oracle_run(cfg, grad: np.ndarray, P_used: int, steps: int, warmup: int, threads: int):
+    """Times the CPU oracle, as it stands, on the first P_used columns of `grad` ([W, ld] host array).
+
+    threads == 1: one call of the oracle's step per iteration.  threads > 1: the column range is split into
+    contiguous pieces and each piece is one call of the same, unchanged oracle step from its own Python
+    thread (the foreign call releases the interpreter lock); every piece redoes the selection, as every
+    parameter-server shard would.  Returns (seconds per step, gradient GB/s)."""
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+
+    W, N = cfg.W, cfg.N
+    ld = grad.shape[1]
+    flat = grad.reshape(-1)
+    theta = np.random.default_rng(cfg.seed).standard_normal(P_used)
+    s0, s1 = np.zeros(P_used), np.zeros(P_used)
+    hyper = {k: float(np.float32(v)) for k, v in cfg.opt.items() if k != "kind"}
+    kind = _oracle_kind(cfg)
+    pieces = column_ranges(P_used, threads)
+
+    def piece(c0, c1, t, arrival, tags):
+        rc, *_ = oracle.step(flat[c0:], c1 - c0, arrival, tags, t, N, cfg.b, theta[c0:c1], s0[c0:c1], s1[c0:c1],
+                             oracle.Opt(kind=kind, step=t + 1, **hyper), ld=ld)
+        return rc
+
     times = []
-    for t in range(warmup + steps):
-        arrival, tags = wl.arrivals(cfg.seed, t, W), wl.tags(cfg.seed, t, W, N)
-        t0 = time.perf_counter()
-        rc, *_ = oracle.step(grad, P_sample, arrival, tags, t, N, cfg.b, theta, s0, s1,
-                             oracle.Opt(kind=kind, step=t + 1, **hyper))
-        dt = time.perf_counter() - t0
-        assert rc == oracle.OK
-        if t >= warmup:
-            times.append(dt)
+    with ThreadPoolExecutor(max_workers=len(pieces)) as pool:
+        for t in range(warmup + steps):
+            arrival, tags = wl.arrivals(cfg.seed, t, W), wl.tags(cfg.seed, t, W, N)
+            t0 = time.perf_counter()
+            if len(pieces) == 1:
+                rcs = [piece(0, P_used, t, arrival, tags)]
+            else:
+                rcs = list(pool.map(lambda r: piece(r[0], r[1], t, arrival, tags), pieces))
+            dt = time.perf_counter() - t0
+            assert all(rc == oracle.OK for rc in rcs)
+            if t >= warmup:
+                times.append(dt)
     sec = float(np.mean(times))
+    esize = grad.dtype.itemsize
+    return sec, N * P_used * esize / sec / 1e9
+
+
+def cpu_baseline(cfg, grad: np.ndarray, P: int, all_steps: int, single_steps: int, warmup: int = 1):
+    """The oracle on all host cores over the first P columns, and on one core over the first quarter of them."""
+    cores = host_cores()
+    sec_all, gbs_all = oracle_run(cfg, grad, P, all_steps, warmup, cores)
+    P_single = max(1, P // 4)
+    sec_one, gbs_one = oracle_run(cfg, grad, P_single, single_steps, warmup, 1)
+    full = P == cfg.P
+    return {
+        "value": gbs_all, "unit": UNIT, "cores": cores, "kind": "oracle", "nproc": os.cpu_count(),
+        "cpu_model": cpu_model(), "ms_per_step": sec_all * 1e3, "full_P": full,
+        "sample": "%s %d columns, all %d rows, %d steps of %.2f s, %d threads each on its own column range"
+                  % ("all" if full else "first", P, cfg.W, all_steps, sec_all, cores),
+        "single_thread": {"value": gbs_one, "unit": UNIT, "cores": 1, "ms_per_step": sec_one * 1e3,
+                          "sample": "first %d of %d columns (1/4), all %d rows, %d steps of %.2f s"
+                                    % (P_single, cfg.P, cfg.W, single_steps, sec_one)},
+    }
+
+
+def workload_config(cfg, P, grad_bytes, total_bytes):
+    """The `config` object of the JSON line; both arms print the same one."""
+    return {"workload": cfg.name, "P": P, "W": cfg.W, "N": cfg.N, "b": cfg.b, "optimizer": cfg.opt["kind"],
+            "grad_dtype": cfg.grad_dtype, "sharding": "one parameter-server column shard of P per GPU",
+            "l2": ("inputs larger than L2 (126 MB): %.3f GB of gradient rows and %.1f MB of parameters and "
+                   "state per step" % (grad_bytes / 1e9, (total_bytes - grad_bytes) / 2e6))
+                  if total_bytes > 4 * 126e6 else
+                  "inputs fit in L2 (%.0f KB per step): a launch-bound workload, read its step time only"
+                  % (total_bytes / 1e3)}
+
+
+def flat_bytes(cfg, P):
     esize = 4 if cfg.grad_dtype == "f32" else 2
-    return sec, N * P_sample * esize / sec / 1e9
+    grad_bytes = cfg.N * P * esize
+    return grad_bytes, grad_bytes + 2 * (1 + N_STATE[cfg.opt["kind"]]) * P * 4
 
 
 def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    P_sample = cfg.P // 4
-    sec, gbs = oracle_sample_run(cfg, P_sample, args.steps, args.warmup)
-    sample = "first %d of %d columns (1/4), all %d rows, %d steps, single thread" % (P_sample, cfg.P, cfg.W, args.steps)
+    P = cfg.P
+    grad = wl.as_oracle_array(wl.grad_matrix(cfg.seed, 0, cfg.W, P, wl.worker_scales(cfg.seed, cfg.W), cfg.grad_dtype, "cpu"))
+    cores = host_cores()
+    sec, gbs = oracle_run(cfg, grad, P, args.steps, args.warmup, cores)
+    sec_one, gbs_one = oracle_run(cfg, grad, max(1, P // 4), max(1, min(args.steps, 3)), min(args.warmup, 1), 1)
+    grad_bytes, total_bytes = flat_bytes(cfg, P)
+    sample = "all %d columns, all %d rows, %d steps, %d threads each on its own column range" % (P, cfg.W, args.steps, cores)
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "P": cfg.P, "W": cfg.W, "N": cfg.N, "b": cfg.b, "optimizer": cfg.opt["kind"],
-                   "grad_dtype": cfg.grad_dtype, "sample": sample},
-        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "config": workload_config(cfg, P, grad_bytes, total_bytes),
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "nproc": os.cpu_count(),
+                         "cpu_model": cpu_model(), "full_P": True, "sample": sample,
+                         "single_thread": {"value": gbs_one, "unit": UNIT, "cores": 1, "ms_per_step": sec_one * 1e3,
+                                           "sample": "first %d of %d columns (1/4)" % (max(1, P // 4), P)}},
         "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
 
+
+# ====================================================================== the five workloads on the GPU
 
 N_STATE = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2, "adagrad": 1}
 N_SETS = 16  # arrival/tag draws rotate, so the kept set differs from step to step
@@ -191,6 +294,49 @@ def selection_sets(cfg, dev):
 def selection_outputs(W, N, dev):
     return (torch.zeros(W, dtype=torch.uint8, device=dev), torch.zeros(N, dtype=torch.int32, device=dev),
             torch.zeros(2, dtype=torch.int32, device=dev))
+
+
+def time_steps(step, steps, warmup):
+    """Mean milliseconds per step over `steps` steps between one pair of CUDA events."""
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(steps):
+        step(warmup + i)
+    stop.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(stop) / steps
+
+
+def time_each_step(step, steps, warmup):
+    """Milliseconds of every single step: an event before the first step and one after each."""
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    marks[0].record()
+    for i in range(steps):
+        step(warmup + i)
+        marks[i + 1].record()
+    torch.cuda.synchronize()
+    return [marks[i].elapsed_time(marks[i + 1]) for i in range(steps)]
+
+
+def spread(ms_list):
+    a = np.asarray(ms_list, dtype=np.float64)
+    return {"steps": int(a.size), "min_ms": float(a.min()), "median_ms": float(np.median(a)),
+            "p95_ms": float(np.percentile(a, 95)), "max_ms": float(a.max())}
+
+
+def rates(total_bytes, grad_bytes, ms):
+    """Throughput figures of one step time against the measured and the nominal HBM peak."""
+    peak, kind = measured_hbm_peak()
+    total = total_bytes / (ms * 1e-3) / 1e9
+    return {"step_us": ms * 1e3, "gradient_gbs": grad_bytes / (ms * 1e-3) / 1e9, "total_gbs": total,
+            "frac_of_%s_peak" % kind: total / peak, "pct_of_nominal_8tbs": 100.0 * total / NOMINAL_HBM_GBS,
+            "algorithmic_bytes_per_step": total_bytes}
 
 
 def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None):
@@ -353,21 +499,64 @@ def setup_arrivals(cfg, dev, sgdb, seed):
         assert c[0] == 0 and c[2] == 0 and c[3] == iteration[0], c
         assert bool(torch.isfinite(theta).all())
 
-    def extra():
-        out = {}
-        for bb in (0, 2, 8):
-            ms = time_steps(make_step(bb), 5, 2)
-            out["b=%d" % bb] = {"ms_per_step": ms, "calls_per_step": N + bb}
-        return {"b_sweep": out, "bytes_per_accepted_arrival": P * 12}
-
     esize = grad.element_size()
     grad_bytes = N * P * esize
     # first accepted row: read row, write acc; middle rows: read row + acc, write acc; N-th: read row + acc + theta
     # + state, write theta + state
     total = grad_bytes + (N - 1) * P * 4 + (N - 1) * P * 4 + 2 * (1 + n_state) * P * 4
+
+    def extra():
+        out = {}
+        for bb in (0, 2, 4, 8):
+            ms = time_steps(make_step(bb), 5, 2)
+            out["b=%d" % bb] = {"ms_per_iteration": ms, "calls_per_iteration": N + bb, "us_per_call": 1e3 * ms / (N + bb),
+                                "us_per_accepted_arrival": 1e3 * ms / N,
+                                "total_gbs": total / (ms * 1e-3) / 1e9}
+        # the batched fused step on the same rows, for comparison
+        mask, order, finfo = selection_outputs(N + 4, N, dev)
+        arr = torch.from_numpy(wl.arrivals(cfg.seed + 4, 0, N + 4)).to(dev)
+        tag = torch.zeros(N + 4, dtype=torch.int32, device=dev)
+
+        def batched(i):
+            opt.step = i + 1
+            sgdb.sgdb_step(grad[: N + 4], P, arr, tag, 0, N, 4, theta, s0, s1, opt, mask, order, finfo)
+
+        ms = time_steps(batched, 10, 3)
+        return {"b_sweep": out, "bytes_per_accepted_arrival": P * 12, "batched_fused_step_ms": ms,
+                "batched_fused_step_total_gbs": (grad_bytes + 2 * (1 + n_state) * P * 4) / (ms * 1e-3) / 1e9}
+
     return dict(step=make_step(cfg.b), check=check, grad_bytes=grad_bytes, total_bytes=total,
                 launches_per_step=N + cfg.b, kernel="accumulate_arrival_kernel<%s, %s>, %d launches per step"
                 % (cfg.grad_dtype, cfg.opt["kind"], N + cfg.b), state=dict(grad=grad), extra=extra)
+
+
+def setup_workload(cfg, dev, sgdb, seed, ema=False, deadline=None):
+    if cfg.segments:
+        return setup_segmented(cfg, dev, sgdb, seed)
+    if cfg.name.startswith("c4"):
+        return setup_arrivals(cfg, dev, sgdb, seed)
+    return setup_flat(cfg, dev, sgdb, seed, ema=ema, deadline=deadline)
+
+
+def other_workload(index, dev, sgdb, steps, warmup):
+    """One of the other seeded workloads, timed on its own: its step time and rates plus the comparison it names."""
+    cfg = wl.CONFIGS[index]
+    wk = setup_workload(cfg, dev, sgdb, cfg.seed)
+    ms = time_each_step(wk["step"], steps, warmup) if index != 0 else [time_steps(wk["step"], steps, warmup)]
+    wk["check"]()
+    out = {"workload": cfg.name, "P": wk.get("P", cfg.P), "W": cfg.W, "N": cfg.N, "b": cfg.b,
+           "optimizer": cfg.opt["kind"], "grad_dtype": cfg.grad_dtype, "kernel": wk["kernel"],
+           "launches_per_step": wk["launches_per_step"]}
+    out.update(rates(wk["total_bytes"], wk["grad_bytes"], float(np.median(ms))))
+    if index == 0:  # 280 KB per step: everything sits in L2, only the time per call means something
+        out = {k: v for k, v in out.items() if not (k.startswith("frac_of") or k.startswith("pct_of") or k.endswith("_gbs"))}
+        out["per_call_us_from_python"] = out["step_us"]
+    else:
+        out["spread"] = spread(ms)
+    extra = wk["extra"]() if callable(wk["extra"]) else wk["extra"]
+    if extra:
+        out.update(extra)
+    return out
 
 
 def max_over_ranks(dist, values, device):
@@ -384,17 +573,9 @@ def whole_job_rate(world: int, bytes_per_rank_step: float, ms_per_step: float) -
     return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
 
 
-def time_steps(step, steps, warmup):
-    for i in range(warmup):
-        step(i)
-    torch.cuda.synchronize()
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record()
-    for i in range(steps):
-        step(warmup + i)
-    stop.record()
-    torch.cuda.synchronize()
-    return start.elapsed_time(stop) / steps
+def release_device_memory():
+    gc.collect()
+    torch.cuda.empty_cache()
 
 
 def run_native(args, cfg):
@@ -419,12 +600,7 @@ def run_native(args, cfg):
         torch.cuda.synchronize()
 
     seed = cfg.seed + 1000 * rank  # every rank is its own parameter-server shard
-    if cfg.segments:
-        wk = setup_segmented(cfg, dev, sgdb, seed)
-    elif cfg.name.startswith("c4"):
-        wk = setup_arrivals(cfg, dev, sgdb, seed)
-    else:
-        wk = setup_flat(cfg, dev, sgdb, seed, ema=args.ema, deadline=args.deadline)
+    wk = setup_workload(cfg, dev, sgdb, seed, ema=args.ema, deadline=args.deadline)
     step = wk["step"]
 
     for i in range(args.warmup):
@@ -441,45 +617,92 @@ def run_native(args, cfg):
     ms_total = start.elapsed_time(stop)
     wk["check"]()
     extra = wk["extra"]() if callable(wk["extra"]) else wk["extra"]
+    extra = dict(extra) if extra else {}
+
+    headline = world == 1 and cfg.name == "c1_inception_rmsprop" and not args.ema and args.deadline is None
+    if headline and not args.only_headline:
+        # ---- spread of single steps, then a sustained run: the server runs for hours, not for 30 ms
+        each = time_each_step(step, args.spread_steps, 3)
+        extra["per_step"] = spread(each)
+        ms_guess = float(np.median(each))
+        n_sustained = max(args.steps, int(np.ceil(args.sustain_seconds * 1e3 / ms_guess)))
+        with ClockSampler(local_rank) as sustained_clocks:
+            ms_sustained = time_steps(step, n_sustained, 3)
+        sc = sustained_clocks.summary()
+        sustained = {"steps": n_sustained, "seconds": ms_sustained * n_sustained * 1e-3, "ms_per_step": ms_sustained,
+                     "clocks": sc}
+        sustained.update({k: v for k, v in rates(wk["total_bytes"], wk["grad_bytes"], ms_sustained).items()
+                          if k != "algorithmic_bytes_per_step"})
+        if sc.get("sm_mhz"):
+            sustained["step_us_times_sm_mhz"] = ms_sustained * 1e3 * sc["sm_mhz"]
+        extra["sustained"] = sustained
+        wk["check"]()
 
     # ---- end to end: gradients start in pinned host memory, new parameters are read back
     flat = not cfg.segments and not cfg.name.startswith("c4")
-    if args.no_e2e or args.ema or args.deadline is not None or not flat or cfg.W * cfg.P * (4 if cfg.grad_dtype == "f32" else 2) > 16e9:
-        return finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, None, 0, clocks)
-    W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
-    st = wk["state"]
-    grad, theta, s0, s1, opt = st["grad"], st["theta"], st["s0"], st["s1"], st["opt"]
-    e2e_steps = max(1, min(args.steps, 3))
-    ws = torch.empty(sgdb.sgdb_step_host_workspace_bytes(grad.dtype, P, P, N, b), dtype=torch.uint8, device=dev)
-    h_grad = torch.empty((W, P), dtype=grad.dtype, pin_memory=True)
-    h_grad.copy_(grad)
-    del grad, st["grad"]
-    h_theta = torch.empty(P, dtype=torch.float32, pin_memory=True)
-    h_mask = torch.empty(W, dtype=torch.uint8, pin_memory=True)
-    h_order = torch.empty(N, dtype=torch.int32, pin_memory=True)
-    h_info = torch.empty(2, dtype=torch.int32, pin_memory=True)
-    h_arr = [torch.from_numpy(wl.arrivals(cfg.seed, t, W)).pin_memory() for t in range(N_SETS)]
-    h_tag = [torch.from_numpy(wl.tags(cfg.seed, t, W, N) - t).pin_memory() for t in range(N_SETS)]
+    e2e_ms, e2e_steps, h_grad = None, 0, None
+    if not (args.no_e2e or args.ema or args.deadline is not None or not flat
+            or cfg.W * cfg.P * (4 if cfg.grad_dtype == "f32" else 2) > 16e9):
+        W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
+        st = wk["state"]
+        grad, theta, s0, s1, opt = st["grad"], st["theta"], st["s0"], st["s1"], st["opt"]
+        e2e_steps = max(1, min(args.steps, 3))
+        ws = torch.empty(sgdb.sgdb_step_host_workspace_bytes(grad.dtype, P, P, N, b), dtype=torch.uint8, device=dev)
+        h_grad = torch.empty((W, P), dtype=grad.dtype, pin_memory=True)
+        h_grad.copy_(grad)
+        del grad, st["grad"]
+        h_theta = torch.empty(P, dtype=torch.float32, pin_memory=True)
+        h_mask = torch.empty(W, dtype=torch.uint8, pin_memory=True)
+        h_order = torch.empty(N, dtype=torch.int32, pin_memory=True)
+        h_info = torch.empty(2, dtype=torch.int32, pin_memory=True)
+        h_arr = [torch.from_numpy(wl.arrivals(cfg.seed, t, W)).pin_memory() for t in range(N_SETS)]
+        h_tag = [torch.from_numpy(wl.tags(cfg.seed, t, W, N) - t).pin_memory() for t in range(N_SETS)]
 
-    def host_step(i):
-        opt.step = i + 1
-        status = sgdb.sgdb_step_host(h_grad, P, h_arr[i % N_SETS], h_tag[i % N_SETS], 0, N, b, theta, s0, s1, opt,
-                                     h_theta, h_mask, h_order, h_info, ws)
-        assert status == 0
+        def host_step(i):
+            opt.step = i + 1
+            status = sgdb.sgdb_step_host(h_grad, P, h_arr[i % N_SETS], h_tag[i % N_SETS], 0, N, b, theta, s0, s1, opt,
+                                         h_theta, h_mask, h_order, h_info, ws)
+            assert status == 0
 
-    host_step(0)
-    barrier()
-    e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e_start.record()
-    for i in range(e2e_steps):
-        host_step(1 + i)
-    e_stop.record()
-    barrier()
-    e2e_ms = e_start.elapsed_time(e_stop)
-    return finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks)
+        host_step(0)
+        barrier()
+        e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e_start.record()
+        for i in range(e2e_steps):
+            host_step(1 + i)
+        e_stop.record()
+        barrier()
+        e2e_ms = e_start.elapsed_time(e_stop)
+        del ws
+
+    # ---- the CPU oracle on this machine's host cores, on the very bytes the GPU consumed
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline and cfg.name.startswith("c1"):
+        if h_grad is None:
+            h_grad = wk["state"]["grad"].cpu()
+        cpu = cpu_baseline(cfg, wl.as_oracle_array(h_grad), cfg.P, all_steps=args.cpu_steps, single_steps=4)
+    del h_grad
+
+    # ---- the other four seeded workloads, one after the other (each frees its memory before the next)
+    if headline and not args.only_headline:
+        del wk["state"], step
+        wk["step"] = wk["check"] = wk["extra"] = None
+        release_device_memory()
+        others = {}
+        for index, name, steps in ((0, "c0", 200), (2, "c2", 20), (3, "c3", 10), (4, "c4", 5)):
+            free, _ = torch.cuda.mem_get_info(dev)
+            need = {0: 1e9, 2: 16e9, 3: 46e9, 4: 12e9}[index]
+            if free < need:
+                others[name] = {"skipped": "needs %.0f GB of free device memory, %.0f GB free" % (need / 1e9, free / 1e9)}
+                continue
+            others[name] = other_workload(index, dev, sgdb, steps, 3)
+            release_device_memory()
+        extra["workloads"] = others
+
+    finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks, cpu)
 
 
-def finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks):
+def finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks, cpu):
     W, N, b = cfg.W, cfg.N, cfg.b
     P = wk.get("P", cfg.P)
     grad_bytes, total_bytes = wk["grad_bytes"], wk["total_bytes"]
@@ -502,24 +725,11 @@ def finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_s
         if (cfg.name == "c1_inception_rmsprop" and not args.ema and args.deadline is None and NCU_TRAFFIC["src_digest"] == digest
                 and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] is not None):
             traffic = NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] * total_bytes
-        cpu = None
-        if world == 1 and not args.no_cpu_baseline and cfg.name.startswith("c1"):
-            P_sample = P // 4
-            sec, gbs = oracle_sample_run(cfg, P_sample, steps=25, warmup=1)
-            cpu = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
-                   "sample": "first %d of %d columns (1/4), all %d rows, 25 steps of %.2f s, single thread"
-                             % (P_sample, P, W, sec)}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": cfg.name, "P": P, "W": W, "N": N, "b": b, "optimizer": cfg.opt["kind"],
-                       "grad_dtype": cfg.grad_dtype, "sharding": "one parameter-server column shard of P per GPU",
-                       "l2": ("inputs larger than L2 (126 MB): %.3f GB of gradient rows and %.1f MB of parameters and "
-                              "state per step" % (grad_bytes / 1e9, (total_bytes - grad_bytes) / 2e6))
-                             if total_bytes > 4 * 126e6 else
-                             "inputs fit in L2 (%.0f KB per step): a launch-bound workload, read its step time only"
-                             % (total_bytes / 1e3)},
+            "vs_baseline": None, "dtype": cfg.grad_dtype, "data": "synthetic",
+            "config": workload_config(cfg, P, grad_bytes, total_bytes),
             "step_us": ms_per_step * 1e3,
             "total_gbs_per_gpu": total_gbs_per_gpu,
             "pct_of_nominal_8tbs": 100.0 * total_gbs_per_gpu / NOMINAL_HBM_GBS,
@@ -546,6 +756,8 @@ def main():
     ap.add_argument("--impl", choices=["native", "reference"], default="native")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--only-headline", action="store_true",
+                    help="skip the spread, the sustained run and the other four workloads (profiling runs)")
     ap.add_argument("--workload", choices=["c0", "c1", "c2", "c3", "c4"], default="c1",
                     help="c1 (default) is the benchmark workload; the others time the remaining seeded workloads")
     ap.add_argument("--ema", action="store_true",
@@ -554,6 +766,9 @@ def main():
                     help="flat workloads: time-out rule (sgdb_step_deadline) with this deadline in seconds")
     ap.add_argument("--columns", type=int, default=0,
                     help="override P with a smaller column count (profiler captures); not the benchmark workload")
+    ap.add_argument("--spread-steps", type=int, default=200, help="single steps timed one by one for the spread")
+    ap.add_argument("--sustain-seconds", type=float, default=2.0, help="length of the sustained run")
+    ap.add_argument("--cpu-steps", type=int, default=5, help="steps of the all-cores oracle leg")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "native":
         args.warmup = 3

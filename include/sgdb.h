@@ -346,6 +346,17 @@ sgdb_status_t sgdb_step_host_static(const void *h_grad, sgdb_dtype_t dt, int64_t
  */
 sgdb_status_t sgdb_set_tuning(int32_t stages, int32_t ctas_per_sm);
 
+/*
+ * sgdb_set_arrival_tuning -- launch-shape knobs of sgdb_accumulate_arrival (no counterpart
+ * in the paper).  resident_bytes: how many leading bytes of the running sum d_acc the
+ * kernels ask the L2 cache to keep between one arrival's launch and the next (the sum is
+ * written by one launch and read by the following one; the gradient rows always stream
+ * through).  0 streams the whole sum; a negative value restores the default.
+ * blocks_per_sm: resident blocks per SM, <= 0 restores the default.  Results do not depend
+ * on either knob.  Affects later calls of this process.
+ */
+sgdb_status_t sgdb_set_arrival_tuning(int64_t resident_bytes, int32_t blocks_per_sm);
+
 const char *sgdb_strerror(sgdb_status_t status); /* static string, never NULL */
 int sgdb_version(void);                          /* major*10000 + minor*100 + patch */
 

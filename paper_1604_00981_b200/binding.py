@@ -26,7 +26,7 @@ _KINDS = {"sgd": SGDB_SGD, "momentum": SGDB_MOMENTUM, "rmsprop": SGDB_RMSPROP, "
 EXPORTS = (
     "sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented",
     "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_accumulate_arrival_ema", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
-    "sgdb_set_tuning", "sgdb_strerror", "sgdb_version",
+    "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version",
 )
 SGDB_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -103,6 +103,7 @@ def _load():
         "sgdb_step_host_static": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt),
                                         vp, vp, vp, vp, vp]),
         "sgdb_set_tuning": (i32, [i32, i32]),
+        "sgdb_set_arrival_tuning": (i32, [i64, i32]),
         "sgdb_strerror": (ctypes.c_char_p, [i32]),
         "sgdb_version": (ctypes.c_int, []),
     }
@@ -164,6 +165,10 @@ def sgdb_version() -> int:
 
 def sgdb_set_tuning(stages: int = 0, ctas_per_sm: int = 0) -> None:
     _check(_lib.sgdb_set_tuning(stages, ctas_per_sm), "sgdb_set_tuning")
+
+
+def sgdb_set_arrival_tuning(resident_bytes: int = -1, blocks_per_sm: int = 0) -> None:
+    _check(_lib.sgdb_set_arrival_tuning(resident_bytes, blocks_per_sm), "sgdb_set_arrival_tuning")
 
 
 def sgdb_select(arrival, tags, t: int, N: int, b: int, mask, order, info, stream=None) -> None:

@@ -50,7 +50,10 @@ struct DeviceInfo {
 DeviceInfo g_dev[kMaxDevices];
 int g_stages = kDefaultStages;
 int g_ctas_per_sm = kDefaultCtasPerSm;
-int g_arrival_blocks_per_sm = 4;
+constexpr int kDefaultArrivalBlocksPerSm = 4;
+constexpr long long kDefaultArrivalResidentBytes = 96ll << 20;
+int g_arrival_blocks_per_sm = kDefaultArrivalBlocksPerSm;
+long long g_arrival_resident_bytes = kDefaultArrivalResidentBytes;
 
 const float kNoDeadline = std::numeric_limits<float>::infinity();
 
@@ -449,6 +452,7 @@ static sgdb_status_t arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag
   if (d_row == nullptr || d_acc == nullptr || d_counter == nullptr || d_theta == nullptr || d_info == nullptr)
     return SGDB_ERR_INVALID_ARG;
   if (!dtype_ok(dt) || N < 1 || P < 0) return SGDB_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_row) % dtype_size(dt) != 0) return SGDB_ERR_INVALID_ARG;
   if (!is_aligned16(d_acc) || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1) ||
       !is_aligned16(d_ema))
     return SGDB_ERR_INVALID_ARG;
@@ -460,10 +464,10 @@ static sgdb_status_t arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag
   st = device_info(&dev);
   if (st != SGDB_OK) return st;
   ArrivalParams p{d_row, row_tag, t, N, P, d_acc, d_counter, d_theta, d_state0, d_state1, d_info,
-                  d_ema, alpha, static_cast<float>(1.0 - static_cast<double>(alpha)), h};
+                  d_ema, alpha, static_cast<float>(1.0 - static_cast<double>(alpha)), g_arrival_resident_bytes / 4, h};
   const int V = dt == SGDB_BF16 ? 8 : 4;
   const long long chunks = (P + V - 1) / V;
-  long long grid = (chunks + 4 * 256 - 1) / (4 * 256);  // 4 chunks per thread and pass
+  long long grid = (chunks + 4 * 256 - 1) / (4 * 256);  // at least 4 chunks per thread
   const long long cap = static_cast<long long>(dev->sms) * g_arrival_blocks_per_sm;
   if (grid > cap) grid = cap;
   if (row_tag != t || grid < 1) grid = 1;  // a wrongly tagged gradient only updates the bookkeeping
@@ -652,6 +656,13 @@ sgdb_status_t sgdb_set_tuning(int32_t stages, int32_t ctas_per_sm) {
   if (stages > 64 || ctas_per_sm > 8) return SGDB_ERR_INVALID_ARG;
   g_stages = stages > 0 ? (stages < 2 ? 2 : stages) : kDefaultStages;
   g_ctas_per_sm = ctas_per_sm > 0 ? ctas_per_sm : kDefaultCtasPerSm;
+  return SGDB_OK;
+}
+
+sgdb_status_t sgdb_set_arrival_tuning(int64_t resident_bytes, int32_t blocks_per_sm) {
+  if (blocks_per_sm > 8) return SGDB_ERR_INVALID_ARG;
+  g_arrival_resident_bytes = resident_bytes >= 0 ? resident_bytes : kDefaultArrivalResidentBytes;
+  g_arrival_blocks_per_sm = blocks_per_sm > 0 ? blocks_per_sm : kDefaultArrivalBlocksPerSm;
   return SGDB_OK;
 }
 

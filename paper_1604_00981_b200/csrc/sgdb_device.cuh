@@ -184,6 +184,68 @@ __device__ __forceinline__ void store_floats(float* p, bool vec, int n, const fl
   }
 }
 
+// The same with an L2 eviction policy chosen by the caller (createpolicy): for data that
+// is read again one launch later and should stay in L2 (evict-last), next to data of the
+// same array that should not (evict-first).
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+  return policy;
+}
+
+__device__ __forceinline__ float4 ld_global_hint(const float4* p, uint64_t policy) {
+  float4 v;
+  asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(p), "l"(policy)
+               : "memory");
+  return v;
+}
+__device__ __forceinline__ float ld_global_hint(const float* p, uint64_t policy) {
+  float v;
+  asm volatile("ld.global.L1::no_allocate.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(v) : "l"(p), "l"(policy) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_global_hint(float4* p, const float4& v, uint64_t policy) {
+  asm volatile("st.global.L1::no_allocate.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(p), "f"(v.x),
+               "f"(v.y), "f"(v.z), "f"(v.w), "l"(policy)
+               : "memory");
+}
+__device__ __forceinline__ void st_global_hint(float* p, float v, uint64_t policy) {
+  asm volatile("st.global.L1::no_allocate.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(p), "f"(v), "l"(policy) : "memory");
+}
+
+template <int V>
+__device__ __forceinline__ void load_floats_hint(const float* p, bool vec, int n, float (&out)[V], uint64_t policy) {
+  if (vec) {
+#pragma unroll
+    for (int q = 0; q < V / 4; ++q) {
+      const float4 v = ld_global_hint(reinterpret_cast<const float4*>(p) + q, policy);
+      out[4 * q + 0] = v.x;
+      out[4 * q + 1] = v.y;
+      out[4 * q + 2] = v.z;
+      out[4 * q + 3] = v.w;
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < V; ++e) out[e] = (e < n) ? ld_global_hint(p + e, policy) : 0.0f;
+  }
+}
+
+template <int V>
+__device__ __forceinline__ void store_floats_hint(float* p, bool vec, int n, const float (&in)[V], uint64_t policy) {
+  if (vec) {
+#pragma unroll
+    for (int q = 0; q < V / 4; ++q)
+      st_global_hint(reinterpret_cast<float4*>(p) + q,
+                     make_float4(in[4 * q + 0], in[4 * q + 1], in[4 * q + 2], in[4 * q + 3]), policy);
+  } else {
+#pragma unroll
+    for (int e = 0; e < V; ++e)
+      if (e < n) st_global_hint(p + e, in[e], policy);
+  }
+}
+
 // ---------------------------------------------------------------- optimizer rules
 
 // One element of the update.  Written with explicit round-to-nearest intrinsics so

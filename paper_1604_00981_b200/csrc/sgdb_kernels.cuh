@@ -570,9 +570,18 @@ struct ArrivalParams {
   int32_t* info;  // [2]
   float* ema;     // optional: average of the parameters, moved when the update fires
   float ema_alpha, ema_one_minus_alpha;
+  long long acc_resident;  // leading elements of acc that are asked to stay in L2 between launches
   Hyper h;
 };
 
+// The running sum is written by one launch and read by the next.  Where it fits, it is kept in
+// L2 across launches: its leading `acc_resident` elements are loaded with an evict-last policy
+// while the gradient row (read once) and the rest of the sum are loaded evict-first; the sum is
+// stored with streaming stores.  (Measured on a B200 at 23.8 M columns: evict-last loads with
+// streaming stores 37 us per launch; evict-last loads and stores 43-49 us; plain stores 55 us;
+// everything streaming 47-50 us.)  The launch that completes the set reads the sum for the last
+// time and releases it (evict-first).  The policies change where the bytes live, never the
+// arithmetic.
 template <typename GT, int EP>
 __global__ void __launch_bounds__(256, 4) accumulate_arrival_kernel(const ArrivalParams p) {
   using Tr = GradTraits<GT>;
@@ -603,6 +612,8 @@ __global__ void __launch_bounds__(256, 4) accumulate_arrival_kernel(const Arriva
     const long long chunks = (p.P + V - 1) / V;
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
     const long long first_chunk = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const uint64_t pol_keep = l2_policy_evict_last();
+    const uint64_t pol_stream = l2_policy_evict_first();
     if (!last) {
       // U chunks per thread and pass, all loads issued before the first use: enough bytes
       // in flight per SM for a stream that reads two arrays and writes one.
@@ -628,7 +639,7 @@ __global__ void __launch_bounds__(256, 4) accumulate_arrival_kernel(const Arriva
 #pragma unroll
               for (int e = 0; e < V; ++e) a[u][e] = 0.0f;
             } else {
-              load_floats<V>(p.acc + i, n[u] == V, n[u], a[u]);
+              load_floats_hint<V>(p.acc + i, n[u] == V, n[u], a[u], i < p.acc_resident ? pol_keep : pol_stream);
             }
           }
         }
@@ -660,7 +671,7 @@ __global__ void __launch_bounds__(256, 4) accumulate_arrival_kernel(const Arriva
 #pragma unroll
           for (int e = 0; e < V; ++e) a[e] = 0.0f;
         } else {
-          load_floats<V>(p.acc + i, vec, n, a);
+          load_floats_hint<V>(p.acc + i, vec, n, a, pol_stream);  // last use of the sum: let it go
         }
         load_floats<V>(p.theta + i, vec, n, th);
         if (Rule::kState0) load_floats<V>(p.s0 + i, vec, n, s0);

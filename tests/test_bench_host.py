@@ -20,8 +20,13 @@ def test_reference_arm_prints_one_contract_line():
     line = json.loads(lines[0])
     assert line["impl"] == "reference" and line["unit"] == "GB/s" and line["higher_is_better"] is True
     assert line["steps"] == 2 and line["warmup"] == 1 and line["value"] > 0 and line["ms_per_step"] > 0
-    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
-    assert line["cpu_baseline"]["value"] == line["value"] == line["e2e"]["value"]
+    cpu = line["cpu_baseline"]
+    assert cpu["kind"] == "oracle" and cpu["cores"] == len(os.sched_getaffinity(0)) and cpu["nproc"] == os.cpu_count()
+    assert isinstance(cpu["cpu_model"], str) and cpu["cpu_model"] and cpu["full_P"] is True
+    assert cpu["single_thread"]["cores"] == 1 and cpu["single_thread"]["value"] > 0
+    assert cpu["value"] == line["value"] == line["e2e"]["value"]
+    # both arms describe the workload with the same keys
+    assert set(line["config"]) == {"workload", "P", "W", "N", "b", "optimizer", "grad_dtype", "sharding", "l2"}
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
     assert line["config"]["workload"].startswith("c1_") and "model" not in line["config"]
     assert line["vs_baseline"] is None and line["gpu_launches"] == 0
@@ -62,3 +67,42 @@ def test_max_over_ranks_and_whole_job_rate_with_two_gloo_ranks(tmp_path):
     # two shards, each moving 8 GB in the slowest rank's 2 ms step: 8 TB/s for the job
     assert bench.whole_job_rate(2, 8e9, 2.0) == 8000.0
     assert bench.max_over_ranks(None, [1.0, 2.0], None) == [1.0, 2.0]
+
+
+def test_column_ranges_cover_every_column_once():
+    sys.path.insert(0, ROOT)
+    import bench
+
+    for P, parts in ((10, 3), (7, 16), (23_800_000, 48), (1, 1)):
+        pieces = bench.column_ranges(P, parts)
+        assert pieces[0][0] == 0 and pieces[-1][1] == P and len(pieces) <= parts
+        assert all(a[1] == b[0] for a, b in zip(pieces, pieces[1:])) and all(c1 > c0 for c0, c1 in pieces)
+
+
+def test_oracle_split_over_threads_equals_one_call():
+    """The all-cores leg of the CPU baseline calls the unchanged oracle step once per column range; the pieces
+    together must give exactly what one call over all columns gives."""
+    sys.path.insert(0, ROOT)
+    import numpy as np
+
+    import bench
+    import oracle
+    from paper_1604_00981_b200 import workload as wl
+
+    cfg = wl.CONFIGS[1]
+    P, W, N = 10_007, cfg.W, cfg.N
+    grad = wl.as_oracle_array(wl.grad_matrix(cfg.seed, 0, W, P, wl.worker_scales(cfg.seed, W), "f32", "cpu"))
+    arrival, tags = wl.arrivals(cfg.seed, 0, W), wl.tags(cfg.seed, 0, W, N)
+    opt = oracle.Opt(kind=oracle.RMSPROP, lr=0.045, decay=0.9, momentum=0.9, eps=1.0)
+    whole = [np.ones(P), np.zeros(P), np.zeros(P)]
+    rc, *_ = oracle.step(grad, P, arrival, tags, 0, N, cfg.b, *whole, opt)
+    assert rc == oracle.OK
+    split = [np.ones(P), np.zeros(P), np.zeros(P)]
+    flat = grad.reshape(-1)
+    for c0, c1 in bench.column_ranges(P, 5):
+        rc, *_ = oracle.step(flat[c0:], c1 - c0, arrival, tags, 0, N, cfg.b, *(a[c0:c1] for a in split), opt, ld=P)
+        assert rc == oracle.OK
+    for a, b in zip(whole, split):
+        assert np.array_equal(a, b)
+    sec, gbs = bench.oracle_run(cfg.__class__(**{**cfg.__dict__, "P": P}), grad, P, steps=1, warmup=0, threads=3)
+    assert sec > 0 and gbs > 0

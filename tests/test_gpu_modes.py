@@ -218,6 +218,84 @@ def test_accumulate_on_arrival(sgdb, cuda_device, kind, dtype, P, b):
         assert x is None or torch.equal(x, y)
 
 
+@pytest.mark.parametrize("side_stream", [False, True])
+@pytest.mark.parametrize("kind,dtype,P", [("rmsprop", "f32", 3_000_001), ("adam", "bf16", 5_000_008)])
+def test_arrivals_enqueued_back_to_back_without_host_reads(sgdb, cuda_device, kind, dtype, P, side_stream):
+    """Whole iterations are enqueued call after call with nothing read back in between, so consecutive launches
+    really follow each other on the device (each launch may be set up while its predecessor still runs; its
+    grid is larger than one wave).  Stale rows, rows arriving after the update and a straggler of the previous
+    iteration are in the sequence.  At the end: parameters, state and the parameter average equal the fused
+    step's bit for bit, and the server counters equal the oracle's replay of the same sequence."""
+    dev = cuda_device
+    N, b, T, seed, alpha = 10, 3, 3, 141, 0.99
+    W = N + b
+    scales = wl.worker_scales(seed, W)
+    theta = wl.theta0(seed, P, dev)
+    theta_f, avg, avg_f = theta.clone(), theta.clone(), theta.clone()
+    s0, s1 = gpu_state(kind, P, dev)
+    sf = gpu_state(kind, P, dev)
+    acc = torch.full((P,), float("nan"), device=dev)
+    counter = torch.zeros(4, dtype=torch.int32, device=dev)
+    info = torch.zeros(2, dtype=torch.int32, device=dev)
+    cols = np.unique(np.concatenate([np.arange(8), np.arange(P - 8, P), np.random.default_rng(seed).integers(0, P, 500)]))
+    cols_d = to_dev(cols, dev)
+    th_o = theta[cols_d].cpu().numpy().astype(np.float64)
+    avg_o = th_o.copy()
+    s0_o, s1_o = oracle_state(kind, len(cols))
+    acc_o, state_o = np.zeros(len(cols)), oracle.new_server_state()
+    stream = torch.cuda.Stream() if side_stream else torch.cuda.current_stream()
+    grads, plans = [], []
+    for t in range(T):  # all inputs first: nothing below this loop touches the host between launches
+        grad = wl.grad_matrix(seed, t, W, P, scales, dtype, dev)
+        arrival, tags = step_inputs(seed, t, W, N)
+        seq = wl.delivery_sequence(arrival)
+        if int((tags == t).sum()) - int(tags[seq[1]] == t) >= N:
+            tags[seq[1]] = t - 1  # an early arrival that is stale
+        grads.append(grad)
+        plans.append((arrival, tags, [int(w) for w in seq]))
+    torch.cuda.synchronize()
+    seen, last_outcome = 0, None
+    with torch.cuda.stream(stream):
+        for t in range(T):
+            arrival, tags, seq = plans[t]
+            opt = gpu_opt(OPTS[kind], t + 1)
+            deliveries = [(grads[t][w], int(tags[w])) for w in seq]
+            if t > 0:  # the gradient the previous iteration dropped last turns up now, tagged t - 1
+                deliveries.insert(2, (grads[t - 1][plans[t - 1][2][-1]], t - 1))
+            for row, tag in deliveries:
+                sgdb.sgdb_accumulate_arrival_ema(row, tag, t, N, acc, counter, theta, s0, s1, opt, avg, alpha, info)
+                seen += 1
+    stream.synchronize()
+    # the oracle's replay of the same sequence (on sampled columns: the bookkeeping does not depend on the data)
+    for t in range(T):
+        arrival, tags, seq = plans[t]
+        sample = wl.as_oracle_array(grads[t].index_select(1, cols_d))
+        deliveries = [(sample[w], int(tags[w])) for w in seq]
+        if t > 0:
+            prev = wl.as_oracle_array(grads[t - 1].index_select(1, cols_d))
+            deliveries.insert(2, (prev[plans[t - 1][2][-1]], t - 1))
+        outcomes = []
+        for row, tag in deliveries:
+            last_outcome = oracle.accumulate_arrival_ema(row, tag, t, N, acc_o, state_o, th_o, s0_o, s1_o,
+                                                         oracle_opt(OPTS[kind], t + 1), avg_o, alpha)
+            outcomes.append(last_outcome)
+        assert outcomes.count(2) == 1 and outcomes.count(1) == N - 1
+    assert counter.cpu().tolist() == [int(state_o[0]), seen, 0, int(state_o[2])] == [0, seen, 0, T]
+    assert info.cpu().tolist() == [last_outcome, int(state_o[0])]
+    # the fused step on the same inputs
+    mask, order, finfo = selection_buffers(W, N, dev)
+    for t in range(T):
+        arrival, tags, _ = plans[t]
+        sgdb.sgdb_step_ema(grads[t], P, to_dev(arrival, dev), to_dev(tags, dev), t, N, b, theta_f, sf[0], sf[1],
+                           gpu_opt(OPTS[kind], t + 1), avg_f, alpha, mask, order, finfo)
+        assert finfo.cpu().tolist()[1] == 0
+    assert torch.equal(theta, theta_f) and torch.equal(avg, avg_f)
+    for x, y in zip((s0, s1), sf):
+        assert x is None or torch.equal(x, y)
+    tol = TOL_F32 if dtype == "f32" else TOL_BF16
+    assert rel_err(theta[cols_d].cpu().numpy(), th_o) < tol and rel_err(avg[cols_d].cpu().numpy(), avg_o) < tol
+
+
 @pytest.mark.parametrize("kind,dtype", [("sgd", "f32"), ("rmsprop", "bf16")])
 def test_asynchronous_server_is_arrival_mode_with_n_equal_one(sgdb, cuda_device, kind, dtype):
     """Algorithm 2 (the asynchronous parameter server) applies each gradient as it arrives.  That is the
