@@ -87,6 +87,8 @@ def _load():
             "oracle_accumulate_arrival_ema",
             "oracle_select_deadline",
             "oracle_step_deadline",
+            "oracle_select_grouped",
+            "oracle_step_grouped",
         ):
             getattr(lib, name).restype = ctypes.c_int
         lib.oracle_ema.restype = None
@@ -275,3 +277,44 @@ def accumulate_arrival_ema(row, row_tag: int, t: int, N: int, acc, state, theta,
     )
     assert rc == OK, rc
     return outcome.value
+
+
+def select_grouped(arrival, tags, group, t: int, M: int, N: int):
+    """Two-level selection: the first N machine messages.  Returns (status, mask[W], group_order[N], order[:n_rows], n_valid)."""
+    arrival = np.ascontiguousarray(arrival, dtype=np.float32)
+    tags = np.ascontiguousarray(tags, dtype=np.int32)
+    group = np.ascontiguousarray(group, dtype=np.int32)
+    W = len(arrival)
+    assert tags.shape == (W,) and group.shape == (W,)
+    mask = np.zeros(W, dtype=np.uint8)
+    group_order = np.full(N, -1, dtype=np.int32)
+    order = np.full(W, -1, dtype=np.int32)
+    n_rows, n_valid = ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = _load().oracle_select_grouped(_p(arrival), _p(tags), _p(group), ctypes.c_int32(t), ctypes.c_int32(W),
+                                       ctypes.c_int32(M), ctypes.c_int32(N), _p(mask), _p(group_order), _p(order),
+                                       ctypes.byref(n_rows), ctypes.byref(n_valid))
+    return rc, mask, group_order, order[: n_rows.value if rc == OK else 0], n_valid.value
+
+
+def step_grouped(grad, P: int, arrival, tags, group, t: int, M: int, N: int, theta, s0, s1, opt: Opt,
+                 ld: int | None = None):
+    """One server iteration over machine messages on fp64 theta/state (in place).
+    Returns (status, mask[W], group_order[N], order[:n_rows], n_valid)."""
+    g, dt = _grad(grad)
+    ld = g.shape[1] if ld is None else ld
+    arrival = np.ascontiguousarray(arrival, dtype=np.float32)
+    tags = np.ascontiguousarray(tags, dtype=np.int32)
+    group = np.ascontiguousarray(group, dtype=np.int32)
+    W = len(arrival)
+    for a in (theta, s0, s1):
+        assert a is None or (a.dtype == np.float64 and a.flags.c_contiguous)
+    mask = np.zeros(W, dtype=np.uint8)
+    group_order = np.full(N, -1, dtype=np.int32)
+    order = np.full(W, -1, dtype=np.int32)
+    n_rows, n_valid = ctypes.c_int32(0), ctypes.c_int32(0)
+    c = opt._c()
+    rc = _load().oracle_step_grouped(
+        _p(g), ctypes.c_int(dt), ctypes.c_int64(P), ctypes.c_int64(ld), _p(arrival), _p(tags), _p(group),
+        ctypes.c_int32(t), ctypes.c_int32(W), ctypes.c_int32(M), ctypes.c_int32(N), _p(theta), _p(s0), _p(s1),
+        ctypes.byref(c), _p(mask), _p(group_order), _p(order), ctypes.byref(n_rows), ctypes.byref(n_valid))
+    return rc, mask, group_order, order[: n_rows.value if rc == OK else 0], n_valid.value

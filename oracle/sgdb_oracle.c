@@ -28,6 +28,9 @@
  *     PARITY UNPINNED BY THE PAPER for momentum / RMSProp / Adam: no equation or
  *     worked number is printed there; the forms below are pinned by closed forms
  *     that hold for the chosen reading only.
+ *   - two-level aggregation (Section 6 names it, nothing more): see oracle_select_grouped.
+ *     PARITY UNPINNED BY THE PAPER; pinned by a replay of machines and messages, by its
+ *     reduction to Algorithm 4 with one worker per machine, and by library means.
  */
 #include <math.h>
 #include <stdint.h>
@@ -321,4 +324,111 @@ int oracle_accumulate_arrival(const void *row, int dtype, int32_t row_tag, int32
     *outcome = 2;
   }
   return ORACLE_OK;
+}
+
+/*
+ * Two-level aggregation.  The paper's conclusion (Section 6) names it in one sentence: the
+ * gradients of workers that share a machine are combined before they are sent to the
+ * parameter server.  It prints no algorithm.  PARITY UNPINNED BY THE PAPER; the reading
+ * taken here keeps Algorithm 4 as it is and lets a machine play the part of a worker:
+ *   - worker w runs on machine group[w], 0 <= group[w] < M;
+ *   - a machine's message is the mean of its workers' gradients (the gradient of its
+ *     combined mini-batch); it can only be sent when the slowest of them is done, so it
+ *     arrives at the maximum of their arrival times;
+ *   - the message counts for iteration t only if every one of its workers computed its
+ *     gradient for t and every arrival time is finite; a machine without workers sends
+ *     nothing;
+ *   - the server runs Algorithm 4 over messages: the first N to arrive are used (equal
+ *     times: lower machine id first), the rest dropped, and theta moves by the mean of the
+ *     N messages.
+ * Outputs: mask [W] 1 for every worker whose gradient is used; group_order [N] the kept
+ * machines in arrival sequence; order [W], of which the first *n_rows entries are the used
+ * workers machine by machine in that sequence and, within a machine, in the order their
+ * gradients were ready (arrival, then id); *n_valid the number of machines whose message
+ * counts.
+ */
+int oracle_select_grouped(const float *arrival, const int32_t *tags, const int32_t *group, int32_t t,
+                          int32_t W, int32_t M, int32_t N, uint8_t *mask, int32_t *group_order,
+                          int32_t *order, int32_t *n_rows, int32_t *n_valid) {
+  if (W < 1 || M < 1 || N < 1) return ORACLE_INVALID;
+  for (int32_t w = 0; w < W; ++w)
+    if (group[w] < 0 || group[w] >= M) return ORACLE_INVALID;
+  float *sent_at = (float *)malloc(sizeof(float) * (size_t)M);
+  int32_t *seq = (int32_t *)malloc(sizeof(int32_t) * (size_t)M);
+  int32_t count = 0;
+  for (int32_t g = 0; g < M; ++g) {
+    int32_t members = 0, counts = 1;
+    float latest = 0.0f;
+    for (int32_t w = 0; w < W; ++w) {
+      if (group[w] != g) continue;
+      if (tags[w] != t || !isfinite(arrival[w])) counts = 0;
+      if (members == 0 || arrival[w] > latest) latest = arrival[w];
+      ++members;
+    }
+    if (members == 0 || !counts) continue;
+    sent_at[g] = latest; /* the machine waits for its slowest worker */
+    int32_t pos = count++;
+    while (pos > 0 && arrives_before(sent_at, g, seq[pos - 1])) {
+      seq[pos] = seq[pos - 1];
+      --pos;
+    }
+    seq[pos] = g;
+  }
+  *n_valid = count;
+  if (count < N) {
+    free(sent_at);
+    free(seq);
+    return ORACLE_INSUFFICIENT;
+  }
+  for (int32_t w = 0; w < W; ++w) mask[w] = 0;
+  int32_t rows = 0;
+  for (int32_t k = 0; k < N; ++k) {
+    int32_t g = seq[k];
+    group_order[k] = g;
+    int32_t first = rows;
+    for (int32_t w = 0; w < W; ++w) {
+      if (group[w] != g) continue;
+      mask[w] = 1;
+      int32_t pos = rows++;
+      while (pos > first && arrives_before(arrival, w, order[pos - 1])) {
+        order[pos] = order[pos - 1];
+        --pos;
+      }
+      order[pos] = w;
+    }
+  }
+  *n_rows = rows;
+  free(sent_at);
+  free(seq);
+  return ORACLE_OK;
+}
+
+/* One server iteration over machine messages: select, form each kept machine's message (the
+ * mean of its workers' gradients), average the N messages, update. */
+int oracle_step_grouped(const void *grad, int dtype, int64_t P, int64_t ld, const float *arrival,
+                        const int32_t *tags, const int32_t *group, int32_t t, int32_t W, int32_t M,
+                        int32_t N, double *theta, double *s0, double *s1, const oracle_opt_t *opt,
+                        uint8_t *mask, int32_t *group_order, int32_t *order, int32_t *n_rows,
+                        int32_t *n_valid) {
+  if (P < 0 || ld < P) return ORACLE_INVALID;
+  int rc = oracle_select_grouped(arrival, tags, group, t, W, M, N, mask, group_order, order, n_rows, n_valid);
+  if (rc != ORACLE_OK) return rc;
+  double *mean = (double *)malloc(sizeof(double) * (size_t)(P > 0 ? P : 1));
+  for (int64_t i = 0; i < P; ++i) {
+    double total = 0.0;
+    for (int32_t k = 0; k < N; ++k) {
+      double message = 0.0;
+      int32_t members = 0;
+      for (int32_t w = 0; w < W; ++w) {
+        if (group[w] != group_order[k]) continue;
+        message += grad_at(grad, dtype, (int64_t)w * ld + i);
+        ++members;
+      }
+      total += message / (double)members;
+    }
+    mean[i] = total / (double)N;
+  }
+  rc = oracle_update(theta, s0, s1, mean, P, opt);
+  free(mean);
+  return rc;
 }

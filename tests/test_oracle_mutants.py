@@ -52,6 +52,18 @@ MUTANTS = [
     ("arrival_counts_stale", "if (row_tag != t || t < state[2] || state[0] >= N) {", "if (t < state[2] || state[0] >= N) {"),
     ("arrival_never_closes", "state[2] = t + 1;", "state[2] = state[2];"),
     ("arrival_divides_late", "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)N;", "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)(N + 1);"),
+    ("machine_sends_at_its_first_worker", "if (members == 0 || arrival[w] > latest) latest = arrival[w];",
+     "if (members == 0 || arrival[w] < latest) latest = arrival[w];"),
+    ("machine_with_a_stale_worker_counts", "if (tags[w] != t || !isfinite(arrival[w])) counts = 0;",
+     "if (!isfinite(arrival[w])) counts = 0;"),
+    ("machine_with_a_missing_worker_counts", "if (tags[w] != t || !isfinite(arrival[w])) counts = 0;",
+     "if (tags[w] != t) counts = 0;"),
+    ("machine_messages_are_sums", "total += message / (double)members;", "total += message;"),
+    ("machine_mean_divides_by_workers", "mean[i] = total / (double)N;", "mean[i] = total / (double)(*n_rows);"),
+    ("machine_without_workers_sends", "if (members == 0 || !counts) continue;", "if (!counts) continue;"),
+    ("machine_rows_in_id_order", "while (pos > first && arrives_before(arrival, w, order[pos - 1])) {", "while (0) {"),
+    ("machine_message_skips_a_worker", "message += grad_at(grad, dtype, (int64_t)w * ld + i);\n        ++members;",
+     "if (members > 0) message += grad_at(grad, dtype, (int64_t)w * ld + i);\n        ++members;"),
     ("arrival_keeps_old_sum", "if (state[0] == 0)\n    for (int64_t i = 0; i < P; ++i) acc[i] = 0.0; /* G = {} */", ""),
 ]
 
@@ -80,7 +92,8 @@ def test_mutant_is_caught_by_a_pin(tmp_path, name, old, new):
                    check=True)
     lib = ctypes.CDLL(str(so_path))
     for fn_name in ("oracle_select", "oracle_aggregate", "oracle_update", "oracle_step", "oracle_accumulate_arrival",
-                    "oracle_step_ema", "oracle_select_deadline", "oracle_step_deadline", "oracle_accumulate_arrival_ema"):
+                    "oracle_step_ema", "oracle_select_deadline", "oracle_step_deadline", "oracle_accumulate_arrival_ema",
+                    "oracle_select_grouped", "oracle_step_grouped"):
         getattr(lib, fn_name).restype = ctypes.c_int
     lib.oracle_ema.restype = None
     lib.oracle_learning_rate.restype = ctypes.c_double

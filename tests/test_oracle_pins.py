@@ -577,3 +577,210 @@ def test_arrival_server_with_average_equals_batched_step_with_average():
                 assert (avg_a == before).all()  # the average only moves when the update fires
         np.testing.assert_allclose(th_a, th_b, rtol=1e-13, atol=1e-14)
         np.testing.assert_allclose(avg_a, avg_b, rtol=1e-13, atol=1e-14)
+
+
+# ---------------------------------------------------------------- two-level aggregation (machines)
+
+
+def test_two_level_hand_worked_iteration():
+    g = _read_golden("two_level_hand_example.txt")
+    t, M, N = int(g["t"][0]), int(g["M"][0]), int(g["N"][0])
+    group = np.array(g["group"], dtype=np.int32)
+    arrival = np.array(g["arrival"], dtype=np.float32)
+    tags = np.array(g["tags"], dtype=np.int32)
+    grad = np.array([g["grad%d" % w] for w in range(len(group))], dtype=np.float32)
+    theta = np.array(g["theta"], dtype=np.float64)
+    rc, mask, group_order, order, n_valid = oracle.step_grouped(grad, 2, arrival, tags, group, t, M, N, theta, None, None,
+                                                                oracle.Opt(kind=oracle.SGD, lr=float(g["lr"][0])))
+    assert rc == oracle.OK and n_valid == int(g["expect_n_valid"][0])
+    assert mask.tolist() == [int(v) for v in g["expect_mask"]]
+    assert group_order.tolist() == [int(v) for v in g["expect_group_order"]]
+    assert order.tolist() == [int(v) for v in g["expect_order"]]
+    assert theta.tolist() == [float(v) for v in g["expect_theta"]]
+
+
+def _replay_machines(arrival, tags, group, t, M, N):
+    """Event by event: workers finish in time order; a machine whose workers are all done sends one message,
+    stamped with that moment; the server takes messages in (time, machine id) order and stops at N.  A machine
+    with a worker that never finishes never sends; one with a worker that computed for another iteration sends
+    a message the server drops.  Returns (kept machine ids in sequence, number of countable messages) or (None, n)."""
+    W = len(arrival)
+    members = {g: [w for w in range(W) if group[w] == g] for g in range(M)}
+    outbox = []
+    for g, ws in members.items():
+        if not ws or not all(math.isfinite(float(arrival[w])) for w in ws):
+            continue
+        clock, done = None, 0
+        for w in sorted(ws, key=lambda w: float(arrival[w])):  # the machine's own workers, one after another
+            clock = float(arrival[w])
+            done += 1
+        assert done == len(ws)
+        outbox.append((clock, g, all(int(tags[w]) == t for w in ws)))
+    outbox.sort(key=lambda m: (m[0], m[1]))
+    kept = []
+    for _, g, current in outbox:
+        if len(kept) == N:
+            break
+        if current:
+            kept.append(g)
+    n_countable = sum(1 for m in outbox if m[2])
+    return (kept if len(kept) == N else None), n_countable
+
+
+def _random_machines(rng, W, M):
+    arrival, tags, t = _random_case(rng, W)
+    group = rng.integers(0, M, size=W).astype(np.int32)
+    return arrival, tags, group, t
+
+
+def test_two_level_selection_matches_replay_of_machines():
+    rng = np.random.default_rng(21)
+    ok = short = 0
+    for trial in range(3000):
+        W, M = int(rng.integers(1, 10)), int(rng.integers(1, 6))
+        N = int(rng.integers(1, M + 1))
+        arrival, tags, group, t = _random_machines(rng, W, M)
+        if trial % 3 == 0:
+            tags[:] = t  # enough cases where most machines count
+        rc, mask, group_order, order, n_valid = oracle.select_grouped(arrival, tags, group, t, M, N)
+        kept, n_countable = _replay_machines(arrival, tags, group, t, M, N)
+        assert n_valid == n_countable
+        if kept is None:
+            assert rc == oracle.INSUFFICIENT
+            short += 1
+            continue
+        ok += 1
+        assert rc == oracle.OK and group_order.tolist() == kept
+        assert mask.tolist() == [1 if group[w] in kept else 0 for w in range(W)]
+        want = []
+        for g in kept:
+            want += sorted([w for w in range(W) if group[w] == g], key=lambda w: (float(arrival[w]), w))
+        assert order.tolist() == want
+    assert ok > 500 and short > 500
+
+
+def test_two_level_kept_machines_are_the_unique_earliest_subset():
+    rng = np.random.default_rng(22)
+    for trial in range(300):
+        W, M = int(rng.integers(2, 10)), int(rng.integers(2, 6))
+        N = int(rng.integers(1, M + 1))
+        arrival, tags, t = _random_case(rng, W, special=False)
+        group = rng.integers(0, M, size=W).astype(np.int32)
+        sent = {}
+        for g in range(M):
+            ws = [w for w in range(W) if group[w] == g]
+            if ws and all(tags[w] == t for w in ws):
+                sent[g] = (max(float(arrival[w]) for w in ws), g)
+        rc, _, group_order, _, n_valid = oracle.select_grouped(arrival, tags, group, t, M, N)
+        assert n_valid == len(sent)
+        if len(sent) < N:
+            assert rc == oracle.INSUFFICIENT
+            continue
+        winners = [sub for sub in itertools.combinations(sorted(sent), N)
+                   if all(sent[a] < sent[r] for a in sub for r in sent if r not in sub)]
+        assert len(winners) == 1 and sorted(group_order.tolist()) == list(winners[0])
+        assert group_order.tolist() == sorted(winners[0], key=lambda g: sent[g])
+
+
+def test_two_level_with_one_worker_per_machine_is_algorithm4():
+    """Machines of one worker each, machine id = worker id: nothing is left of the second level, and the result
+    must be Algorithm 4's own, bit for bit, for every rule."""
+    rng = np.random.default_rng(23)
+    for kind in (oracle.SGD, oracle.MOMENTUM, oracle.RMSPROP, oracle.ADAM, oracle.ADAGRAD):
+        for trial in range(20):
+            W = int(rng.integers(1, 9))
+            N = int(rng.integers(1, W + 1))
+            P = 5
+            arrival, tags, t = _random_case(rng, W)
+            grad = rng.standard_normal((W, P)).astype(np.float32)
+            opt = oracle.Opt(kind=kind, lr=0.1, momentum=0.9, decay=0.9, beta1=0.9, beta2=0.99, eps=0.5, step=3)
+            a = [rng.standard_normal(P), np.abs(rng.standard_normal(P)), np.abs(rng.standard_normal(P))]
+            b = [x.copy() for x in a]
+            rc1, mask1, order1, n1 = oracle.step(grad, P, arrival, tags, t, N, W - N, *a, opt)
+            rc2, mask2, gorder2, order2, n2 = oracle.step_grouped(grad, P, arrival, tags, np.arange(W, dtype=np.int32), t,
+                                                                  W, N, *b, opt)
+            assert rc1 == rc2 and n1 == n2
+            for x, y in zip(a, b):
+                assert np.array_equal(x, y)
+            if rc1 == oracle.OK:
+                assert mask1.tolist() == mask2.tolist() and order1.tolist() == order2.tolist() == gorder2.tolist()
+
+
+def test_two_level_with_equal_machines_is_the_mean_over_their_workers():
+    """Equal machine sizes: the mean of the machines' means is numpy's mean over all workers of the kept machines."""
+    rng = np.random.default_rng(24)
+    M, per, N, P = 6, 4, 4, 33
+    W = M * per
+    group = rng.permutation(np.repeat(np.arange(M), per)).astype(np.int32)  # workers of a machine need not be neighbours
+    arrival = rng.lognormal(0.0, 0.3, W).astype(np.float32)
+    tags = np.full(W, 2, np.int32)
+    grad = rng.standard_normal((W, P)).astype(np.float32)
+    theta = rng.standard_normal(P)
+    theta0 = theta.copy()
+    rc, mask, group_order, order, n_valid = oracle.step_grouped(grad, P, arrival, tags, group, 2, M, N, theta, None, None,
+                                                                oracle.Opt(kind=oracle.SGD, lr=0.25))
+    assert rc == oracle.OK and n_valid == M and int(mask.sum()) == N * per == len(order)
+    sent = [max(arrival[group == g]) for g in range(M)]
+    assert group_order.tolist() == list(np.argsort(np.array(sent, np.float32), kind="stable")[:N])
+    want = theta0 - 0.25 * np.mean(grad[np.isin(group, group_order)].astype(np.float64), axis=0)
+    assert np.allclose(theta, want, rtol=0, atol=1e-15)
+
+
+def test_two_level_unequal_machines_weigh_messages_equally_and_wait_for_the_slowest():
+    """Constant rows of powers of two: the mean of the kept machines' means is exact, and differs from the mean
+    over workers, from a sum of machine sums and from what a send-at-first-worker rule would keep."""
+    group = np.array([0, 0, 0, 0, 1, 2, 2], np.int32)
+    arrival = np.array([0.1, 0.2, 0.3, 9.0, 1.0, 0.5, 2.0], np.float32)  # machine 0 has an early start and a late finish
+    tags = np.zeros(7, np.int32)
+    consts = np.array([1, 2, 4, 8, 16, 32, 64], np.float64)
+    grad = np.repeat(consts[:, None], 3, axis=1).astype(np.float32)
+    theta = np.zeros(3)
+    rc, mask, group_order, order, _ = oracle.step_grouped(grad, 3, arrival, tags, group, 0, 3, 2, theta, None, None,
+                                                          oracle.Opt(kind=oracle.SGD, lr=1.0))
+    assert rc == oracle.OK and group_order.tolist() == [1, 2] and order.tolist() == [4, 5, 6]
+    assert mask.tolist() == [0, 0, 0, 0, 1, 1, 1]
+    assert theta.tolist() == [-(16 + (32 + 64) / 2) / 2] * 3  # = -32, not -(16+32+64)/3 and not -(16+96)
+
+
+def test_two_level_a_stale_or_missing_worker_silences_its_machine():
+    rng = np.random.default_rng(25)
+    M, per, N, P = 5, 3, 3, 4
+    W = M * per
+    group = np.repeat(np.arange(M), per).astype(np.int32)
+    arrival = (1.0 + np.arange(W) * 0.125).astype(np.float32)  # machine g sends before machine g + 1
+    tags = np.full(W, 7, np.int32)
+    grad = rng.standard_normal((W, P)).astype(np.float32)
+    base = oracle.select_grouped(arrival, tags, group, 7, M, N)
+    assert base[0] == oracle.OK and base[2].tolist() == [0, 1, 2] and base[4] == M
+    for spoil in ("stale", "future", "nan", "inf"):
+        a, tg = arrival.copy(), tags.copy()
+        if spoil == "stale":
+            tg[4] = 6
+        elif spoil == "future":
+            tg[4] = 8
+        elif spoil == "nan":
+            a[4] = np.nan
+        else:
+            a[4] = np.inf
+        rc, mask, group_order, order, n_valid = oracle.select_grouped(a, tg, group, 7, M, N)
+        assert rc == oracle.OK and n_valid == M - 1 and group_order.tolist() == [0, 2, 3]  # machine 1 is out, 3 moves up
+        assert mask.tolist() == [1 if g in (0, 2, 3) else 0 for g in group]
+    # rows of machines that are not used cannot influence the result
+    theta_a, theta_b = np.ones(P), np.ones(P)
+    poisoned = grad.copy()
+    poisoned[group >= 3] = np.nan
+    opt = oracle.Opt(kind=oracle.SGD, lr=0.5)
+    assert oracle.step_grouped(grad, P, arrival, tags, group, 7, M, N, theta_a, None, None, opt)[0] == oracle.OK
+    assert oracle.step_grouped(poisoned, P, arrival, tags, group, 7, M, N, theta_b, None, None, opt)[0] == oracle.OK
+    assert np.array_equal(theta_a, theta_b) and np.isfinite(theta_a).all()
+    # too few countable messages: nothing moves; a machine id out of range is refused
+    tags[::per] = 6
+    before = theta_a.copy()
+    rc, *_ , n_valid = oracle.step_grouped(grad, P, arrival, tags, group, 7, M, N, theta_a, None, None, opt)
+    assert rc == oracle.INSUFFICIENT and n_valid == 0 and np.array_equal(theta_a, before)
+    bad = group.copy()
+    bad[0] = M
+    assert oracle.select_grouped(arrival, np.full(W, 7, np.int32), bad, 7, M, N)[0] == oracle.INVALID
+    # a machine without workers sends nothing
+    rc, _, group_order, _, n_valid = oracle.select_grouped(arrival[:6], np.full(6, 7, np.int32), np.array([0, 0, 0, 2, 2, 2], np.int32), 7, 3, 2)
+    assert rc == oracle.OK and n_valid == 2 and group_order.tolist() == [0, 2]
