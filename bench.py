@@ -339,7 +339,7 @@ def rates(total_bytes, grad_bytes, ms):
             "algorithmic_bytes_per_step": total_bytes}
 
 
-def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None):
+def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
     """Workloads with one flat parameter vector (tiny SGD, Inception-sized RMSProp, large bf16 Adam)."""
     W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
     scales = wl.worker_scales(cfg.seed, W)
@@ -360,9 +360,21 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None):
                 for t in range(N_SETS)]
         kept_mean = float(np.mean(kept))
 
+    if machines:  # two-level: worker w runs on machine w * machines // W; as many machines are kept as hold N workers
+        group = torch.from_numpy((np.arange(W) * machines // W).astype(np.int32)).to(dev)
+        n_machines = max(1, N * machines // W)
+        group_order = torch.zeros(n_machines, dtype=torch.int32, device=dev)
+        order = torch.zeros(W, dtype=torch.int32, device=dev)
+        info = torch.zeros(3, dtype=torch.int32, device=dev)
+        tag_d = [torch.zeros(W, dtype=torch.int32, device=dev)] * N_SETS  # every worker current: all machines count
+        kept_mean = n_machines * W / machines  # exact when the machines are equally large
+
     def step(i):
         opt.step = i + 1
-        if deadline is not None:
+        if machines:
+            sgdb.sgdb_step_grouped(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], group, 0, machines, n_machines, theta, s0,
+                                   s1, opt, mask, group_order, order, info)
+        elif deadline is not None:
             sgdb.sgdb_step_deadline(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, deadline, 1, theta, s0, s1, opt,
                                     mask, order, info)
         elif ema:  # the step plus the running average of the parameters (last line of the server's loop)
@@ -420,8 +432,10 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None):
     total = grad_bytes + 2 * (1 + n_state) * P * 4 + (2 * P * 4 if ema else 0)
     return dict(step=step, check=check, grad_bytes=grad_bytes, total_bytes=total,
                 launches_per_step=1, kernel="stream_rows_kernel<%s, %s>%s (the step is this one launch)"
-                % (cfg.grad_dtype, cfg.opt["kind"], " + parameter average" if ema else ""), state=state,
-                extra={"parameter_average": True} if ema else
+                % (cfg.grad_dtype, cfg.opt["kind"], " + parameter average" if ema else
+                   (", two-level: %d machines, %d kept" % (machines, n_machines) if machines else "")), state=state,
+                extra={"parameter_average": True} if ema else {"machines": machines, "machines_kept": n_machines,
+                                                               "rows_used": kept_mean} if machines else
                 ({"deadline_s": deadline, "mean_rows_kept": kept_mean} if deadline is not None else
                  (graph_replay if P * W <= 1_000_000 else separate_calls)))
 
@@ -530,12 +544,12 @@ def setup_arrivals(cfg, dev, sgdb, seed):
                 % (cfg.grad_dtype, cfg.opt["kind"], N + cfg.b), state=dict(grad=grad), extra=extra)
 
 
-def setup_workload(cfg, dev, sgdb, seed, ema=False, deadline=None):
+def setup_workload(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
     if cfg.segments:
         return setup_segmented(cfg, dev, sgdb, seed)
     if cfg.name.startswith("c4"):
         return setup_arrivals(cfg, dev, sgdb, seed)
-    return setup_flat(cfg, dev, sgdb, seed, ema=ema, deadline=deadline)
+    return setup_flat(cfg, dev, sgdb, seed, ema=ema, deadline=deadline, machines=machines)
 
 
 def other_workload(index, dev, sgdb, steps, warmup):
@@ -600,7 +614,7 @@ def run_native(args, cfg):
         torch.cuda.synchronize()
 
     seed = cfg.seed + 1000 * rank  # every rank is its own parameter-server shard
-    wk = setup_workload(cfg, dev, sgdb, seed, ema=args.ema, deadline=args.deadline)
+    wk = setup_workload(cfg, dev, sgdb, seed, ema=args.ema, deadline=args.deadline, machines=args.machines)
     step = wk["step"]
 
     for i in range(args.warmup):
@@ -619,7 +633,8 @@ def run_native(args, cfg):
     extra = wk["extra"]() if callable(wk["extra"]) else wk["extra"]
     extra = dict(extra) if extra else {}
 
-    headline = world == 1 and cfg.name == "c1_inception_rmsprop" and not args.ema and args.deadline is None
+    headline = (world == 1 and cfg.name == "c1_inception_rmsprop" and not args.ema and args.deadline is None
+                and not args.machines)
     if headline and not args.only_headline:
         # ---- spread of single steps, then a sustained run: the server runs for hours, not for 30 ms
         each = time_each_step(step, args.spread_steps, 3)
@@ -641,7 +656,7 @@ def run_native(args, cfg):
     # ---- end to end: gradients start in pinned host memory, new parameters are read back
     flat = not cfg.segments and not cfg.name.startswith("c4")
     e2e_ms, e2e_steps, h_grad = None, 0, None
-    if not (args.no_e2e or args.ema or args.deadline is not None or not flat
+    if not (args.no_e2e or args.ema or args.deadline is not None or args.machines or not flat
             or cfg.W * cfg.P * (4 if cfg.grad_dtype == "f32" else 2) > 16e9):
         W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
         st = wk["state"]
@@ -722,7 +737,7 @@ def finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_s
         peak, peak_kind = measured_hbm_peak()
         digest = kernel_source_digest()
         traffic = None
-        if (cfg.name == "c1_inception_rmsprop" and not args.ema and args.deadline is None and NCU_TRAFFIC["src_digest"] == digest
+        if (cfg.name == "c1_inception_rmsprop" and not args.ema and args.deadline is None and not args.machines and NCU_TRAFFIC["src_digest"] == digest
                 and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] is not None):
             traffic = NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] * total_bytes
         line = {
@@ -764,6 +779,8 @@ def main():
                     help="flat workloads: also keep the exponential moving average of the parameters (sgdb_step_ema)")
     ap.add_argument("--deadline", type=float, default=None,
                     help="flat workloads: time-out rule (sgdb_step_deadline) with this deadline in seconds")
+    ap.add_argument("--machines", type=int, default=0,
+                    help="flat workloads: two-level aggregation (sgdb_step_grouped) with the workers spread over this many machines")
     ap.add_argument("--columns", type=int, default=0,
                     help="override P with a smaller column count (profiler captures); not the benchmark workload")
     ap.add_argument("--spread-steps", type=int, default=200, help="single steps timed one by one for the spread")

@@ -237,6 +237,42 @@ sgdb_status_t sgdb_step_segmented(const sgdb_segment_t *d_segments, int32_t S, s
                                   int32_t *d_order, int32_t *d_info, void *stream);
 
 /*
+ * sgdb_select_grouped, sgdb_step_grouped -- two-level aggregation: the gradients of workers
+ * that share a machine are combined before they reach the server.  The paper names this in
+ * its conclusion (Section 6) and prints no algorithm; here a machine takes a worker's place
+ * in Algorithm 4 (Section 3 for the first-N rule):
+ *   - worker w runs on machine d_group[w], 0 <= d_group[w] < M;
+ *   - a machine's message is the mean of its workers' gradients and arrives when the
+ *     slowest of them does (the maximum of their arrival times);
+ *   - the message counts for iteration t only if every worker of the machine is tagged t
+ *     and has a finite arrival time; a machine without workers sends nothing;
+ *   - the server uses the first N messages to arrive (equal times: lower machine id) and
+ *     moves theta by the mean of those N messages; rows of machines it drops are never read.
+ *
+ *   d_arrival, d_tags, d_group [W]   per worker;  W, M <= SGDB_MAX_WORKERS, 1 <= N <= M
+ *   d_mask        [W] uint8  out: 1 for every worker whose gradient is used
+ *   d_group_order [N] int32  out: the kept machines in the order their messages arrived
+ *   d_order       [W] int32  out: the used workers in summation sequence -- machine by
+ *                            machine in that order, within a machine by (arrival, id);
+ *                            d_info[2] entries are written
+ *   d_info        [3] int32  out: {machines whose message counts, status, workers used}
+ * Summation: a machine's rows are added one after another from +0 and divided by their
+ * number; the N messages are added one after another from +0 and divided by N (fp32).  The
+ * result has the bits of sgdb_aggregate per machine followed by sgdb_step over the machines'
+ * means.  With fewer than N messages that count, d_info[1] = SGDB_ERR_INSUFFICIENT and nothing
+ * else is touched; a machine id outside [0, M) gives d_info[1] = SGDB_ERR_INVALID_ARG likewise.
+ * sgdb_step_grouped is one launch.
+ */
+sgdb_status_t sgdb_select_grouped(const float *d_arrival, const int32_t *d_tags, const int32_t *d_group,
+                                  int32_t t, int32_t W, int32_t M, int32_t N, uint8_t *d_mask,
+                                  int32_t *d_group_order, int32_t *d_order, int32_t *d_info, void *stream);
+sgdb_status_t sgdb_step_grouped(const void *d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld,
+                                const float *d_arrival, const int32_t *d_tags, const int32_t *d_group,
+                                int32_t t, int32_t W, int32_t M, int32_t N, float *d_theta, float *d_state0,
+                                float *d_state1, const sgdb_opt_t *opt, uint8_t *d_mask,
+                                int32_t *d_group_order, int32_t *d_order, int32_t *d_info, void *stream);
+
+/*
  * sgdb_accumulate_arrival -- Algorithm 4's inner loop taken literally: one
  * gradient per call, in the order the gradients reach the server.
  *

@@ -26,7 +26,7 @@ _KINDS = {"sgd": SGDB_SGD, "momentum": SGDB_MOMENTUM, "rmsprop": SGDB_RMSPROP, "
 EXPORTS = (
     "sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented",
     "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_accumulate_arrival_ema", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
-    "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version",
+    "sgdb_select_grouped", "sgdb_step_grouped", "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version",
 )
 SGDB_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -94,6 +94,9 @@ def _load():
         "sgdb_ema": (i32, [vp, vp, i64, ctypes.c_float, vp, vp]),
         "sgdb_learning_rate": (ctypes.c_double, [ctypes.c_double, ctypes.c_double, i64, i64, ctypes.c_double]),
         "sgdb_step_segmented": (i32, [vp, i32, i32, vp, vp, i32, i32, i32, ctypes.POINTER(_COpt), vp, vp, vp, vp]),
+        "sgdb_select_grouped": (i32, [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]),
+        "sgdb_step_grouped": (i32, [vp, i32, i64, i64, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt),
+                                    vp, vp, vp, vp, vp]),
         "sgdb_accumulate_arrival": (i32, [vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, ctypes.POINTER(_COpt), vp, vp]),
         "sgdb_accumulate_arrival_ema": (i32, [vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, ctypes.POINTER(_COpt), vp,
                                               ctypes.c_float, vp, vp]),
@@ -280,6 +283,31 @@ def sgdb_step_segmented(table, S: int, grad_dtype, arrival, tags, t: int, N: int
                                     t, N, b, ctypes.byref(c), _dev(mask, torch.uint8, "mask"),
                                     _dev(order, torch.int32, "order"), _dev(info, torch.int32, "info"),
                                     _stream(stream)), "sgdb_step_segmented")
+
+
+def sgdb_select_grouped(arrival, tags, group, t: int, M: int, N: int, mask, group_order, order, info, stream=None) -> None:
+    """Two-level selection: the first N machine messages.  mask u8[W], group_order i32[N], order i32[W], info i32[3]."""
+    W = arrival.numel()
+    _check(_lib.sgdb_select_grouped(_dev(arrival, torch.float32, "arrival"), _dev(tags, torch.int32, "tags"),
+                                    _dev(group, torch.int32, "group"), t, W, M, N, _dev(mask, torch.uint8, "mask"),
+                                    _dev(group_order, torch.int32, "group_order"), _dev(order, torch.int32, "order"),
+                                    _dev(info, torch.int32, "info"), _stream(stream)), "sgdb_select_grouped")
+
+
+def sgdb_step_grouped(grad, P: int, arrival, tags, group, t: int, M: int, N: int, theta, state0, state1, opt: Opt,
+                      mask, group_order, order, info, ld: int | None = None, stream=None) -> None:
+    """One fused iteration over machine messages: machines send the mean of their workers' rows, the first N
+    messages are averaged, then the optimizer rule."""
+    ld = grad.stride(0) if ld is None else ld
+    W = arrival.numel()
+    c = opt._c()
+    _check(_lib.sgdb_step_grouped(_dev(grad, None, "grad"), _grad_dtype(grad), P, ld,
+                                  _dev(arrival, torch.float32, "arrival"), _dev(tags, torch.int32, "tags"),
+                                  _dev(group, torch.int32, "group"), t, W, M, N, _dev(theta, torch.float32, "theta"),
+                                  _dev(state0, torch.float32, "state0"), _dev(state1, torch.float32, "state1"),
+                                  ctypes.byref(c), _dev(mask, torch.uint8, "mask"),
+                                  _dev(group_order, torch.int32, "group_order"), _dev(order, torch.int32, "order"),
+                                  _dev(info, torch.int32, "info"), _stream(stream)), "sgdb_step_grouped")
 
 
 def sgdb_accumulate_arrival(row, row_tag: int, t: int, N: int, acc, counter, theta, state0, state1,

@@ -8,6 +8,7 @@
 #include <cstdio>
 #include <cstring>
 #include <limits>
+#include <atomic>
 #include <mutex>
 
 #include "sgdb_kernels.cuh"
@@ -44,6 +45,7 @@ constexpr int kDefaultCtasPerSm = 2;
 
 struct DeviceInfo {
   bool known = false;
+  int index = 0;
   int sms = 0;
   int max_smem_optin = 0;
 };
@@ -69,6 +71,7 @@ sgdb_status_t device_info(const DeviceInfo** out) {
         cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) !=
             cudaSuccess)
       return SGDB_ERR_CUDA;
+    d.index = dev;
     d.known = true;
   }
   *out = &d;
@@ -151,20 +154,21 @@ sgdb_status_t check_selection_args(const void* arrival, const void* tags, int32_
 
 // ---------------------------------------------------------------- row-streaming launch
 
-template <typename GT, int EP>
-sgdb_status_t launch_stream_t(const StreamParams& p_in, long long total_tiles_hint, cudaStream_t stream) {
+template <typename GT, int EP, bool GROUPED = false>
+sgdb_status_t launch_stream_t(const StreamParams& p_in, cudaStream_t stream) {
   const DeviceInfo* dev = nullptr;
   sgdb_status_t st = device_info(&dev);
   if (st != SGDB_OK) return st;
   StreamParams p = p_in;
   constexpr int kCH = Shape<GT>::kCH;
   constexpr int kStageBytes = kNT * kCH * 16;
-  auto kernel = stream_rows_kernel<GT, EP, kNT, kCH>;
+  auto kernel = stream_rows_kernel<GT, EP, kNT, kCH, GROUPED>;
 
-  // shared memory: ring + 2 barriers per slot + order[N] + tile prefix[S + 1]
+  // shared memory: ring + 2 barriers per slot + order[N] + tile prefix[S + 1] + selection scratch
   if (p.order_cap < p.N) p.order_cap = p.N;
   const size_t fixed = static_cast<size_t>((p.order_cap + 3) & ~3) * 4 + (p.table ? (static_cast<size_t>(p.S) + 1) * 4 : 0) +
-                       (p.arrival ? static_cast<size_t>(p.W) * 4 : 0) + 16;
+                       (p.arrival ? static_cast<size_t>(p.W) * 4 : 0) +
+                       (GROUPED ? (4 * static_cast<size_t>(p.M) + static_cast<size_t>(p.N) + 1) * 4 : 0) + 16;
   int ctas_per_sm = g_ctas_per_sm;
   int stages = g_stages;
   const size_t per_sm_budget = static_cast<size_t>(dev->max_smem_optin);
@@ -175,37 +179,57 @@ sgdb_status_t launch_stream_t(const StreamParams& p_in, long long total_tiles_hi
   const size_t smem = static_cast<size_t>(stages) * (kStageBytes + 16) + fixed;
   if (smem > per_sm_budget) return SGDB_ERR_UNSUPPORTED;
   p.stages = stages;
-  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
-      cudaSuccess)
-    return launch_status();
+  // the opt-in to large dynamic shared memory is kept per kernel and device: asked for again only when a
+  // launch needs more than any launch of this kernel before it
+  static std::atomic<int> smem_allowed[kMaxDevices];
+  if (static_cast<int>(smem) > smem_allowed[dev->index].load(std::memory_order_relaxed)) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
+        cudaSuccess)
+      return launch_status();
+    smem_allowed[dev->index].store(static_cast<int>(smem), std::memory_order_relaxed);
+  }
   long long grid = static_cast<long long>(dev->sms) * ctas_per_sm;
   if (p.table == nullptr) {
     const long long tile = static_cast<long long>(kNT) * kCH * GradTraits<GT>::kVec;
     p.total_tiles = static_cast<int>((p.flat.len + tile - 1) / tile);
     if (p.total_tiles < grid) grid = p.total_tiles;
   }
-  (void)total_tiles_hint;
   if (grid < 1) grid = 1;
   kernel<<<static_cast<unsigned>(grid), kNT + 32, smem, stream>>>(p);
   return launch_status();
 }
 
 template <typename GT>
-sgdb_status_t launch_stream_ep(int ep, const StreamParams& p, long long tiles, cudaStream_t stream) {
+sgdb_status_t launch_stream_ep(int ep, const StreamParams& p, cudaStream_t stream) {
   switch (ep) {
-    case EP_MEAN: return launch_stream_t<GT, EP_MEAN>(p, tiles, stream);
-    case EP_SGD: return launch_stream_t<GT, EP_SGD>(p, tiles, stream);
-    case EP_MOMENTUM: return launch_stream_t<GT, EP_MOMENTUM>(p, tiles, stream);
-    case EP_RMSPROP: return launch_stream_t<GT, EP_RMSPROP>(p, tiles, stream);
-    case EP_ADAM: return launch_stream_t<GT, EP_ADAM>(p, tiles, stream);
-    case EP_ADAGRAD: return launch_stream_t<GT, EP_ADAGRAD>(p, tiles, stream);
+    case EP_MEAN: return launch_stream_t<GT, EP_MEAN>(p, stream);
+    case EP_SGD: return launch_stream_t<GT, EP_SGD>(p, stream);
+    case EP_MOMENTUM: return launch_stream_t<GT, EP_MOMENTUM>(p, stream);
+    case EP_RMSPROP: return launch_stream_t<GT, EP_RMSPROP>(p, stream);
+    case EP_ADAM: return launch_stream_t<GT, EP_ADAM>(p, stream);
+    case EP_ADAGRAD: return launch_stream_t<GT, EP_ADAGRAD>(p, stream);
   }
   return SGDB_ERR_INVALID_ARG;
 }
 
-sgdb_status_t launch_stream(int dt, int ep, const StreamParams& p, long long tiles, cudaStream_t stream) {
-  return dt == SGDB_BF16 ? launch_stream_ep<BF16>(ep, p, tiles, stream)
-                         : launch_stream_ep<float>(ep, p, tiles, stream);
+sgdb_status_t launch_stream(int dt, int ep, const StreamParams& p, cudaStream_t stream) {
+  return dt == SGDB_BF16 ? launch_stream_ep<BF16>(ep, p, stream) : launch_stream_ep<float>(ep, p, stream);
+}
+
+template <typename GT>
+sgdb_status_t launch_stream_grouped_ep(int ep, const StreamParams& p, cudaStream_t stream) {
+  switch (ep) {
+    case EP_SGD: return launch_stream_t<GT, EP_SGD, true>(p, stream);
+    case EP_MOMENTUM: return launch_stream_t<GT, EP_MOMENTUM, true>(p, stream);
+    case EP_RMSPROP: return launch_stream_t<GT, EP_RMSPROP, true>(p, stream);
+    case EP_ADAM: return launch_stream_t<GT, EP_ADAM, true>(p, stream);
+    case EP_ADAGRAD: return launch_stream_t<GT, EP_ADAGRAD, true>(p, stream);
+  }
+  return SGDB_ERR_INVALID_ARG;
+}
+
+sgdb_status_t launch_stream_grouped(int dt, int ep, const StreamParams& p, cudaStream_t stream) {
+  return dt == SGDB_BF16 ? launch_stream_grouped_ep<BF16>(ep, p, stream) : launch_stream_grouped_ep<float>(ep, p, stream);
 }
 
 long long tiles_of(int dt, long long len) {
@@ -285,7 +309,7 @@ sgdb_status_t sgdb_aggregate(const void* d_grad, sgdb_dtype_t dt, int64_t P, int
   StreamParams p = flat_params(d_mean, nullptr, nullptr, d_grad, ld, P, N);  // the mean goes where theta would
   p.order = d_order;
   p.info = d_info;
-  return launch_stream(dt, EP_MEAN, p, tiles_of(dt, P), static_cast<cudaStream_t>(stream));
+  return launch_stream(dt, EP_MEAN, p, static_cast<cudaStream_t>(stream));
 }
 
 sgdb_status_t sgdb_update(float* d_theta, float* d_state0, float* d_state1, const float* d_mean, int64_t P,
@@ -341,7 +365,7 @@ static sgdb_status_t step_flat(const void* d_grad, sgdb_dtype_t dt, int64_t P, i
   p.ema_alpha = alpha;
   p.ema_one_minus_alpha = static_cast<float>(1.0 - static_cast<double>(alpha));
   p.h = h;
-  return launch_stream(dt, ep, p, tiles_of(dt, P), s);  // one launch: selection is the kernel's prologue
+  return launch_stream(dt, ep, p, s);  // one launch: selection is the kernel's prologue
 }
 
 sgdb_status_t sgdb_step(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, const float* d_arrival,
@@ -417,7 +441,7 @@ sgdb_status_t sgdb_step_deadline(const void* d_grad, sgdb_dtype_t dt, int64_t P,
   p.keep_all = true;
   p.order_cap = W;
   p.h = h;
-  return launch_stream(dt, ep, p, tiles_of(dt, P), static_cast<cudaStream_t>(stream));
+  return launch_stream(dt, ep, p, static_cast<cudaStream_t>(stream));
 }
 
 sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, sgdb_dtype_t dt,
@@ -443,7 +467,57 @@ sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, s
   p.N = N;
   set_in_kernel_selection(&p, d_arrival, d_tags, t, N + b, d_mask, d_order, d_info);
   p.h = h;
-  return launch_stream(dt, ep, p, 0, s);
+  return launch_stream(dt, ep, p, s);
+}
+
+static sgdb_status_t check_grouped_args(const void* arrival, const void* tags, const void* group, int32_t W, int32_t M,
+                                        int32_t N, const void* mask, const void* group_order, const void* order,
+                                        const void* info) {
+  if (arrival == nullptr || tags == nullptr || group == nullptr || mask == nullptr || group_order == nullptr ||
+      order == nullptr || info == nullptr)
+    return SGDB_ERR_INVALID_ARG;
+  if (W < 1 || M < 1 || N < 1 || N > M) return SGDB_ERR_INVALID_ARG;
+  if (W > SGDB_MAX_WORKERS || M > SGDB_MAX_WORKERS) return SGDB_ERR_INVALID_ARG;
+  return SGDB_OK;
+}
+
+sgdb_status_t sgdb_select_grouped(const float* d_arrival, const int32_t* d_tags, const int32_t* d_group, int32_t t,
+                                  int32_t W, int32_t M, int32_t N, uint8_t* d_mask, int32_t* d_group_order,
+                                  int32_t* d_order, int32_t* d_info, void* stream) {
+  sgdb_status_t st = check_grouped_args(d_arrival, d_tags, d_group, W, M, N, d_mask, d_group_order, d_order, d_info);
+  if (st != SGDB_OK) return st;
+  const int larger = W > M ? W : M;
+  const int threads = (larger + 31) & ~31;
+  select_grouped_kernel<<<1, threads, 0, static_cast<cudaStream_t>(stream)>>>(d_arrival, d_tags, d_group, t, N, W, M,
+                                                                              d_mask, d_group_order, d_order, d_info);
+  return launch_status();
+}
+
+sgdb_status_t sgdb_step_grouped(const void* d_grad, sgdb_dtype_t dt, int64_t P, int64_t ld, const float* d_arrival,
+                                const int32_t* d_tags, const int32_t* d_group, int32_t t, int32_t W, int32_t M,
+                                int32_t N, float* d_theta, float* d_state0, float* d_state1, const sgdb_opt_t* opt,
+                                uint8_t* d_mask, int32_t* d_group_order, int32_t* d_order, int32_t* d_info,
+                                void* stream) {
+  sgdb_status_t st = check_grouped_args(d_arrival, d_tags, d_group, W, M, N, d_mask, d_group_order, d_order, d_info);
+  if (st != SGDB_OK) return st;
+  st = check_flat(d_grad, dt, P, ld, N);
+  if (st != SGDB_OK) return st;
+  Hyper h;
+  int ep = 0;
+  st = prepare_rule(opt, d_state0, d_state1, &h, &ep);
+  if (st != SGDB_OK) return st;
+  if (d_theta == nullptr || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
+    return SGDB_ERR_INVALID_ARG;
+  if (P == 0)
+    return sgdb_select_grouped(d_arrival, d_tags, d_group, t, W, M, N, d_mask, d_group_order, d_order, d_info, stream);
+  StreamParams p = flat_params(d_theta, d_state0, d_state1, d_grad, ld, P, N);
+  set_in_kernel_selection(&p, d_arrival, d_tags, t, W, d_mask, d_order, d_info);
+  p.order_cap = W;
+  p.group = d_group;
+  p.M = M;
+  p.group_order_out = d_group_order;
+  p.h = h;
+  return launch_stream_grouped(dt, ep, p, static_cast<cudaStream_t>(stream));
 }
 
 static sgdb_status_t arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag, int32_t t, int32_t N, int64_t P,
@@ -595,7 +669,7 @@ sgdb_status_t sgdb_step_host(const void* h_grad, sgdb_dtype_t dt, int64_t P, int
     p.info = d_info;
     p.status_out = d_info + 1;
     p.h = h;
-    st = launch_stream(dt, ep, p, tiles_of(dt, P), s);
+    st = launch_stream(dt, ep, p, s);
     if (st != SGDB_OK) return st;
     if (h_theta_out != nullptr &&
         cudaMemcpyAsync(h_theta_out, d_theta, static_cast<size_t>(P) * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)

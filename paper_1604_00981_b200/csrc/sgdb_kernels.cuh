@@ -105,6 +105,172 @@ __global__ void __launch_bounds__(1024) select_first_n_kernel(const float* __res
   block_select(arrival, tags, t, N, W, deadline, keep_all, s_key, s_order, &s_count, true, mask, order, info);
 }
 
+// ---------------------------------------------------------------------- two-level selection
+//
+// Workers share machines: group[w] in [0, M).  A machine's message counts when the machine
+// has at least one worker and every one of its workers is valid (tag == t, finite arrival); it
+// arrives when its slowest worker does.  Machines are ranked like workers above, by (message
+// arrival, machine id); the first N are kept.  The rows that will be added are the workers of
+// the kept machines, machine by machine in message order and, within a machine, in (arrival,
+// id) order: s_order[gend[r] .. gend[r + 1]) are the rows of the machine of rank r.
+//
+// Finite floats are mapped to unsigned integers of the same order so that the latest arrival
+// of a machine is one shared-memory atomicMax per worker; 0 is below every mapped value.
+__device__ __forceinline__ unsigned ordered_bits(float a) {
+  const unsigned u = __float_as_uint(a);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(unsigned u) {
+  return __uint_as_float((u & 0x80000000u) ? (u ^ 0x80000000u) : ~u);
+}
+
+// Inclusive scan of a[1..n] in place by the first warp (a[0] stays): a[i] <- a[1] + ... + a[i].
+__device__ __forceinline__ void warp_scan_in_place(int* a, int n) {
+  const int lane = threadIdx.x & 31;
+  int carry = 0;
+  for (int base = 1; base <= n; base += 32) {
+    const int idx = base + lane;
+    int v = idx <= n ? a[idx] : 0;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, v, d);
+      if (lane >= d) v += up;
+    }
+    v += carry;
+    if (idx <= n) a[idx] = v;
+    carry = __shfl_sync(0xffffffffu, v, 31);
+  }
+}
+
+//   s_key [W] floats, s_order [W] ints, s_gkey [M] words, s_gcnt / s_gbad / s_grank [M] ints,
+//   s_gend [N + 1] ints, s_count [2] ints; global outputs are written only when `writer`.
+// Returns the number of rows to add (s_order holds that many, s_gend their split by machine), or
+// 0 when fewer than N machines count or a machine id is out of range; then only g_info is written:
+// {machines that count, status, rows used}.
+__device__ __forceinline__ int block_select_grouped(const float* __restrict__ arrival, const int32_t* __restrict__ tags,
+                                                    const int32_t* __restrict__ group, int32_t t, int32_t N, int32_t W,
+                                                    int32_t M, float* s_key, int* s_order, unsigned* s_gkey,
+                                                    int* s_gcnt, int* s_gbad, int* s_grank, int* s_gend, int* s_count,
+                                                    bool writer, uint8_t* __restrict__ g_mask,
+                                                    int32_t* __restrict__ g_group_order, int32_t* __restrict__ g_order,
+                                                    int32_t* __restrict__ g_info) {
+  const int tid = threadIdx.x;
+  const int nthreads = blockDim.x;
+  for (int g = tid; g < M; g += nthreads) {
+    s_gkey[g] = 0u;
+    s_gcnt[g] = 0;
+    s_gbad[g] = 0;
+  }
+  if (tid == 0) {
+    s_count[0] = 0;  // machines that count
+    s_count[1] = 0;  // a machine id out of range was seen
+  }
+  __syncthreads();
+  for (int w = tid; w < W; w += nthreads) {
+    const int g = group[w];
+    const float a = arrival[w];
+    s_key[w] = a;
+    if (g < 0 || g >= M) {
+      s_count[1] = 1;
+    } else if (tags[w] == t && isfinite(a)) {
+      atomicMax(&s_gkey[g], ordered_bits(a));
+      atomicAdd(&s_gcnt[g], 1);
+    } else {
+      s_gbad[g] = 1;
+    }
+  }
+  __syncthreads();
+  if (s_count[1] != 0) {
+    if (writer && tid == 0) {
+      g_info[0] = 0;
+      g_info[1] = SGDB_ERR_INVALID_ARG;
+      g_info[2] = 0;
+    }
+    return 0;
+  }
+  float* s_gtime = reinterpret_cast<float*>(s_gkey);  // same words, now the message's arrival time
+  const int m_end = (M + 31) & ~31;
+  for (int g = tid; g < m_end; g += nthreads) {
+    bool counts = false;
+    if (g < M) {
+      counts = s_gcnt[g] > 0 && s_gbad[g] == 0;
+      s_gtime[g] = counts ? from_ordered_bits(s_gkey[g]) : __int_as_float(0x7fc00000);
+    }
+    const unsigned votes = __ballot_sync(0xffffffffu, counts);
+    if ((tid & 31) == 0 && votes != 0) atomicAdd(&s_count[0], __popc(votes));
+  }
+  __syncthreads();
+  const int n_valid = s_count[0];
+  const bool enough = n_valid >= N;
+  if (!enough) {
+    if (writer && tid == 0) {
+      g_info[0] = n_valid;
+      g_info[1] = SGDB_ERR_INSUFFICIENT;
+      g_info[2] = 0;
+    }
+    return 0;
+  }
+  for (int g = tid; g < M; g += nthreads) {
+    const float a = s_gtime[g];
+    int rank = 0;
+#pragma unroll 8
+    for (int j = 0; j < M; ++j) {
+      const float aj = s_gtime[j];
+      rank += ((aj < a) || (aj == a && j < g)) ? 1 : 0;
+    }
+    const bool kept = (a == a) && rank < N;
+    s_grank[g] = kept ? rank : -1;
+    if (kept) {
+      s_gend[rank + 1] = s_gcnt[g];
+      if (writer) g_group_order[rank] = g;
+    }
+  }
+  if (tid == 0) s_gend[0] = 0;
+  __syncthreads();
+  if (tid < 32) warp_scan_in_place(s_gend, N);
+  __syncthreads();
+  for (int w = tid; w < W; w += nthreads) {
+    const int g = group[w];
+    const int r = s_grank[g];
+    if (r >= 0) {
+      const float a = s_key[w];
+      int before = 0;
+      for (int j = 0; j < W; ++j) {
+        const float aj = s_key[j];
+        before += (group[j] == g && ((aj < a) || (aj == a && j < w))) ? 1 : 0;
+      }
+      const int pos = s_gend[r] + before;
+      s_order[pos] = w;
+      if (writer) g_order[pos] = w;
+    }
+    if (writer) g_mask[w] = r >= 0 ? 1 : 0;
+  }
+  __syncthreads();
+  const int n_rows = s_gend[N];
+  if (writer && tid == 0) {
+    g_info[0] = n_valid;
+    g_info[1] = SGDB_OK;
+    g_info[2] = n_rows;
+  }
+  return n_rows;
+}
+
+__global__ void __launch_bounds__(1024) select_grouped_kernel(const float* __restrict__ arrival,
+                                                              const int32_t* __restrict__ tags,
+                                                              const int32_t* __restrict__ group, int32_t t, int32_t N,
+                                                              int32_t W, int32_t M, uint8_t* __restrict__ mask,
+                                                              int32_t* __restrict__ group_order,
+                                                              int32_t* __restrict__ order, int32_t* __restrict__ info) {
+  __shared__ float s_key[SGDB_MAX_WORKERS];
+  __shared__ int s_order[SGDB_MAX_WORKERS];
+  __shared__ unsigned s_gkey[SGDB_MAX_WORKERS];
+  __shared__ int s_gcnt[SGDB_MAX_WORKERS], s_gbad[SGDB_MAX_WORKERS], s_grank[SGDB_MAX_WORKERS];
+  __shared__ int s_gend[SGDB_MAX_WORKERS + 1];
+  __shared__ int s_count[2];
+  block_select_grouped(arrival, tags, group, t, N, W, M, s_key, s_order, s_gkey, s_gcnt, s_gbad, s_grank, s_gend, s_count,
+                       true, mask, group_order, order, info);
+}
+
 // ====================================================================== row streaming
 //
 // Persistent blocks walk over column tiles of TILE = NT*CH*V columns.  For a tile,
@@ -146,6 +312,11 @@ struct StreamParams {
   uint8_t* mask_out;
   int32_t* order_out;
   int32_t* info_out;
+  // Two-level aggregation (GROUPED kernels): worker w runs on machine group[w] in [0, M); N counts
+  // machines, W workers; the kept machines go to group_order_out [N], info_out has 3 words.
+  const int32_t* group;
+  int32_t M;
+  int32_t* group_order_out;
   // Optional (flat case): exponential moving average of the parameters, updated in the
   // same pass from the value theta had BEFORE this step's update.
   float* ema;
@@ -212,7 +383,9 @@ __device__ __forceinline__ TileDesc<GT> locate_tile(const StreamParams& p, const
   return td;
 }
 
-template <typename GT, int EP, int NT, int CH>
+// GROUPED: the kept rows fall into runs (one per kept machine); every run is summed on its own,
+// divided by its length, and the runs' means are added in sequence and divided by their number.
+template <typename GT, int EP, int NT, int CH, bool GROUPED = false>
 __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamParams p) {
   using Tr = GradTraits<GT>;
   using Rule = RuleTraits<EP>;
@@ -234,12 +407,27 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
   int* order_s = reinterpret_cast<int*>(empty_bar + stages);
   int* prefix_s = order_s + ((p.order_cap + 3) & ~3);
   float* key_s = reinterpret_cast<float*>(prefix_s + (p.table != nullptr ? p.S + 1 : 0));
+  int* gend_s = nullptr;  // GROUPED: rows of the machine of rank r are order_s[gend_s[r] .. gend_s[r + 1])
+  int n_div = N;          // what the sum is divided by in the end
 
-  if (p.arrival != nullptr) {
+  if constexpr (GROUPED) {
+    unsigned* gkey_s = reinterpret_cast<unsigned*>(key_s + p.W);
+    int* gcnt_s = reinterpret_cast<int*>(gkey_s + p.M);
+    int* gbad_s = gcnt_s + p.M;
+    int* grank_s = gbad_s + p.M;
+    gend_s = grank_s + p.M;
+    __shared__ int s_gcount[2];
+    N = block_select_grouped(p.arrival, p.tags, p.group, p.t, p.N, p.W, p.M, key_s, order_s, gkey_s, gcnt_s, gbad_s,
+                             grank_s, gend_s, s_gcount, blockIdx.x == 0, p.mask_out, p.group_order_out, p.order_out,
+                             p.info_out);
+    if (N == 0) return;
+    n_div = p.N;
+  } else if (p.arrival != nullptr) {
     // fewer than N current gradients: the iteration cannot complete, nothing is touched
     N = block_select(p.arrival, p.tags, p.t, N, p.W, p.deadline, p.keep_all, key_s, order_s, &s_count,
                      blockIdx.x == 0, p.mask_out, p.order_out, p.info_out);
     if (N == 0) return;
+    n_div = N;
   } else {
     if (p.info != nullptr && p.info[1] != SGDB_OK) return;
     for (int i = tid; i < N; i += NT + 32) order_s[i] = p.order[i];
@@ -318,7 +506,7 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
     }
   } else {
     // ------------------------------------------------------------ consumers
-    const float n_as_float = static_cast<float>(N);
+    const float n_as_float = static_cast<float>(n_div);
     int s = 0;
     uint32_t phase = 0;
     for (int tile = blockIdx.x; tile < total_tiles && !timed_out; tile += gridDim.x) {
@@ -347,12 +535,15 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
       const bool has_tail = td.bulk_cols < td.ncols;
 
       if (td.bad) continue;  // reported by block 0 in the prologue
-      if (td.bulk_cols == 0) {
-        for (int k = 0; k < N; ++k) add_row_tail(k);
-      } else {
-        int k = 0;
+
+      // adds rows order_s[k .. k_end) into acc, in that sequence; false when a wait ran out
+      auto add_rows = [&](int k, const int k_end) -> bool {
+        if (td.bulk_cols == 0) {
+          for (; k < k_end; ++k) add_row_tail(k);
+          return true;
+        }
         // two rows per pass: both slots are waited for and read before the dependent adds
-        for (; k + 1 < N; k += 2) {
+        for (; k + 1 < k_end; k += 2) {
           const int sa = s;
           const uint32_t pa = phase;
           if (++s == stages) {
@@ -365,10 +556,7 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
             s = 0;
             phase ^= 1u;
           }
-          if (!mbar_wait(full_addr + 8u * sa, pa, &s_abort) || !mbar_wait(full_addr + 8u * sb, pb, &s_abort)) {
-            timed_out = true;
-            break;
-          }
+          if (!mbar_wait(full_addr + 8u * sa, pa, &s_abort) || !mbar_wait(full_addr + 8u * sb, pb, &s_abort)) return false;
           const unsigned char* stage_a = smem + static_cast<size_t>(sa) * STAGE_BYTES;
           const unsigned char* stage_b = smem + static_cast<size_t>(sb) * STAGE_BYTES;
           uint4 va[CH], vb[CH];
@@ -403,31 +591,58 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
             add_row_tail(k + 1);
           }
         }
-        if (!timed_out && k < N) {  // N odd: the last row on its own
-          if (!mbar_wait(full_addr + 8u * s, phase, &s_abort)) {
-            timed_out = true;
-          } else {
-            const unsigned char* stage = smem + static_cast<size_t>(s) * STAGE_BYTES;
+        if (k < k_end) {  // an odd count: the last row on its own
+          if (!mbar_wait(full_addr + 8u * s, phase, &s_abort)) return false;
+          const unsigned char* stage = smem + static_cast<size_t>(s) * STAGE_BYTES;
 #pragma unroll
-            for (int c = 0; c < CH; ++c) {
-              const int o = (tid + c * NT) * V;
-              if (o + V <= td.bulk_cols) {
-                const uint4 v = *reinterpret_cast<const uint4*>(stage + static_cast<size_t>(o) * sizeof(GT));
-                float x[V];
-                Tr::unpack(v, x);
+          for (int c = 0; c < CH; ++c) {
+            const int o = (tid + c * NT) * V;
+            if (o + V <= td.bulk_cols) {
+              const uint4 v = *reinterpret_cast<const uint4*>(stage + static_cast<size_t>(o) * sizeof(GT));
+              float x[V];
+              Tr::unpack(v, x);
 #pragma unroll
-                for (int e = 0; e < V; ++e) acc[c][e] = __fadd_rn(acc[c][e], x[e]);
-              }
+              for (int e = 0; e < V; ++e) acc[c][e] = __fadd_rn(acc[c][e], x[e]);
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_addr + 8u * s);
-            if (++s == stages) {
-              s = 0;
-              phase ^= 1u;
-            }
-            if (has_tail) add_row_tail(k);
           }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty_addr + 8u * s);
+          if (++s == stages) {
+            s = 0;
+            phase ^= 1u;
+          }
+          if (has_tail) add_row_tail(k);
         }
+        return true;
+      };
+
+      if constexpr (GROUPED) {
+        float total[CH][V];
+#pragma unroll
+        for (int c = 0; c < CH; ++c)
+#pragma unroll
+          for (int e = 0; e < V; ++e) total[c][e] = 0.0f;
+        for (int r = 0; r < n_div; ++r) {
+          const int k0 = gend_s[r], k1 = gend_s[r + 1];
+          if (!add_rows(k0, k1)) {
+            timed_out = true;
+            break;
+          }
+          const float members = static_cast<float>(k1 - k0);
+#pragma unroll
+          for (int c = 0; c < CH; ++c)
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+              total[c][e] = __fadd_rn(total[c][e], __fdiv_rn(acc[c][e], members));  // this machine's message
+              acc[c][e] = 0.0f;
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < CH; ++c)
+#pragma unroll
+          for (int e = 0; e < V; ++e) acc[c][e] = total[c][e];
+      } else {
+        if (!add_rows(0, N)) timed_out = true;
       }
       if (timed_out) break;
 
