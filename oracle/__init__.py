@@ -87,6 +87,8 @@ def _load():
             "oracle_accumulate_arrival_ema",
             "oracle_select_deadline",
             "oracle_step_deadline",
+            "oracle_accumulate_arrival_deadline",
+            "oracle_accumulate_close",
             "oracle_select_grouped",
             "oracle_step_grouped",
         ):
@@ -318,3 +320,26 @@ def step_grouped(grad, P: int, arrival, tags, group, t: int, M: int, N: int, the
         ctypes.c_int32(t), ctypes.c_int32(W), ctypes.c_int32(M), ctypes.c_int32(N), _p(theta), _p(s0), _p(s1),
         ctypes.byref(c), _p(mask), _p(group_order), _p(order), ctypes.byref(n_rows), ctypes.byref(n_valid))
     return rc, mask, group_order, order[: n_rows.value if rc == OK else 0], n_valid.value
+
+
+def accumulate_arrival_deadline(row, row_tag: int, row_arrival: float, t: int, deadline: float, acc, state) -> int:
+    """Time-out rule, one received gradient: joins the set iff tagged t, t open, arrived by the deadline.  0 dropped, 1 added."""
+    r, dt = _grad(row)
+    assert acc.dtype == np.float64 and state.dtype == np.int32 and len(state) == 3
+    outcome = ctypes.c_int32(-1)
+    rc = _load().oracle_accumulate_arrival_deadline(
+        _p(r), ctypes.c_int(dt), ctypes.c_int32(row_tag), ctypes.c_float(row_arrival), ctypes.c_int32(t),
+        ctypes.c_float(deadline), ctypes.c_int64(len(acc)), _p(acc), _p(state), ctypes.byref(outcome))
+    assert rc == OK, rc
+    return outcome.value
+
+
+def accumulate_close(t: int, n_min: int, acc, state, theta, s0, s1, opt: Opt, avg=None, alpha: float = 0.0):
+    """The deadline of iteration t has passed.  Returns (status, outcome): outcome 2 = theta updated with the mean of the
+    set, 0 = nothing done; status INSUFFICIENT (nothing changed) with fewer than n_min gradients in the set."""
+    outcome = ctypes.c_int32(-1)
+    c = opt._c()
+    rc = _load().oracle_accumulate_close(
+        ctypes.c_int32(t), ctypes.c_int32(n_min), ctypes.c_int64(len(theta)), _p(acc), _p(state), _p(theta), _p(s0), _p(s1),
+        ctypes.byref(c), _p(avg), ctypes.c_double(alpha), ctypes.byref(outcome))
+    return rc, outcome.value

@@ -432,3 +432,51 @@ int oracle_step_grouped(const void *grad, int dtype, int64_t P, int64_t ld, cons
   free(mean);
   return rc;
 }
+
+/*
+ * The time-out rule (see oracle_select_deadline) one received gradient at a time.  The server
+ * listens until `deadline`: a gradient joins the set iff it is tagged t, iteration t is still
+ * open and it arrived (finite time) by the deadline; there is no upper count.  When the
+ * deadline has passed the server closes the iteration (oracle_accumulate_close): with at least
+ * n_min gradients in the set it moves theta by their mean (divisor: the number in the set),
+ * empties the set and opens t + 1; with fewer the iteration does not complete and nothing
+ * changes.  state as in oracle_accumulate_arrival.  PARITY UNPINNED BY THE PAPER, like the
+ * batched time-out rule it must agree with.
+ * *outcome: 0 dropped, 1 added.
+ */
+int oracle_accumulate_arrival_deadline(const void *row, int dtype, int32_t row_tag, float row_arrival,
+                                       int32_t t, float deadline, int64_t P, double *acc,
+                                       int32_t *state, int32_t *outcome) {
+  if (P < 0) return ORACLE_INVALID;
+  state[1] += 1;
+  if (row_tag != t || t < state[2] || !isfinite(row_arrival) || !(row_arrival <= deadline)) {
+    *outcome = 0;
+    return ORACLE_OK;
+  }
+  if (state[0] == 0)
+    for (int64_t i = 0; i < P; ++i) acc[i] = 0.0; /* G = {} */
+  for (int64_t i = 0; i < P; ++i) acc[i] += grad_at(row, dtype, i);
+  state[0] += 1;
+  *outcome = 1;
+  return ORACLE_OK;
+}
+
+/* The deadline of iteration t has passed.  *outcome: 2 theta updated, 0 nothing done (t was closed
+ * already).  Returns ORACLE_INSUFFICIENT, with nothing changed, when fewer than n_min gradients are
+ * in the set.  avg may be NULL; otherwise it takes in theta as it was before the update. */
+int oracle_accumulate_close(int32_t t, int32_t n_min, int64_t P, double *acc, int32_t *state,
+                            double *theta, double *s0, double *s1, const oracle_opt_t *opt,
+                            double *avg, double alpha, int32_t *outcome) {
+  if (n_min < 1 || P < 0) return ORACLE_INVALID;
+  *outcome = 0;
+  if (t < state[2]) return ORACLE_OK;
+  if (state[0] < n_min) return ORACLE_INSUFFICIENT;
+  if (avg != NULL) oracle_ema(avg, theta, P, alpha); /* theta is still theta(t) here */
+  for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)state[0];
+  int rc = oracle_update(theta, s0, s1, acc, P, opt);
+  if (rc != ORACLE_OK) return rc;
+  state[0] = 0;
+  state[2] = t + 1;
+  *outcome = 2;
+  return ORACLE_OK;
+}

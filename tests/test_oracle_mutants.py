@@ -64,6 +64,14 @@ MUTANTS = [
     ("machine_rows_in_id_order", "while (pos > first && arrives_before(arrival, w, order[pos - 1])) {", "while (0) {"),
     ("machine_message_skips_a_worker", "message += grad_at(grad, dtype, (int64_t)w * ld + i);\n        ++members;",
      "if (members > 0) message += grad_at(grad, dtype, (int64_t)w * ld + i);\n        ++members;"),
+    ("arrival_deadline_strict", "|| !isfinite(row_arrival) || !(row_arrival <= deadline)) {", "|| !isfinite(row_arrival) || !(row_arrival < deadline)) {"),
+    ("arrival_deadline_ignored", "|| !isfinite(row_arrival) || !(row_arrival <= deadline)) {", "|| !isfinite(row_arrival)) {"),
+    ("arrival_deadline_counts_stale", "if (row_tag != t || t < state[2] || !isfinite(row_arrival)", "if (t < state[2] || !isfinite(row_arrival)"),
+    ("close_divides_by_n_min", "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)state[0];", "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)n_min;"),
+    ("close_ignores_n_min", "if (state[0] < n_min) return ORACLE_INSUFFICIENT;", "if (state[0] < 1) return ORACLE_INSUFFICIENT;"),
+    ("close_leaves_iteration_open", "state[0] = 0;\n  state[2] = t + 1;\n  *outcome = 2;\n  return ORACLE_OK;\n}\n", "state[0] = 0;\n  *outcome = 2;\n  return ORACLE_OK;\n}\n"),
+    ("close_averages_updated_parameters", "if (avg != NULL) oracle_ema(avg, theta, P, alpha); /* theta is still theta(t) here */\n  for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)state[0];\n  int rc = oracle_update(theta, s0, s1, acc, P, opt);\n  if (rc != ORACLE_OK) return rc;",
+     "for (int64_t i = 0; i < P; ++i) acc[i] = acc[i] / (double)state[0];\n  int rc = oracle_update(theta, s0, s1, acc, P, opt);\n  if (rc != ORACLE_OK) return rc;\n  if (avg != NULL) oracle_ema(avg, theta, P, alpha);"),
     ("arrival_keeps_old_sum", "if (state[0] == 0)\n    for (int64_t i = 0; i < P; ++i) acc[i] = 0.0; /* G = {} */", ""),
 ]
 
@@ -93,7 +101,7 @@ def test_mutant_is_caught_by_a_pin(tmp_path, name, old, new):
     lib = ctypes.CDLL(str(so_path))
     for fn_name in ("oracle_select", "oracle_aggregate", "oracle_update", "oracle_step", "oracle_accumulate_arrival",
                     "oracle_step_ema", "oracle_select_deadline", "oracle_step_deadline", "oracle_accumulate_arrival_ema",
-                    "oracle_select_grouped", "oracle_step_grouped"):
+                    "oracle_select_grouped", "oracle_step_grouped", "oracle_accumulate_arrival_deadline", "oracle_accumulate_close"):
         getattr(lib, fn_name).restype = ctypes.c_int
     lib.oracle_ema.restype = None
     lib.oracle_learning_rate.restype = ctypes.c_double

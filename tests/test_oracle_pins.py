@@ -784,3 +784,80 @@ def test_two_level_a_stale_or_missing_worker_silences_its_machine():
     # a machine without workers sends nothing
     rc, _, group_order, _, n_valid = oracle.select_grouped(arrival[:6], np.full(6, 7, np.int32), np.array([0, 0, 0, 2, 2, 2], np.int32), 7, 3, 2)
     assert rc == oracle.OK and n_valid == 2 and group_order.tolist() == [0, 2]
+
+
+# ---------------------------------------------------------------- time-out rule, one gradient at a time
+
+
+@pytest.mark.parametrize("kind", [oracle.SGD, oracle.RMSPROP])
+def test_arrival_server_with_deadline_equals_batched_deadline_step(kind):
+    """Gradients delivered one by one in arrival sequence (stale ones, late ones and a straggler of the previous
+    iteration included), then the close call: same set, same divisor, same bits as the batched time-out step, which
+    is pinned on its own above.  Also in event order (late rows delivered after the close)."""
+    rng = np.random.default_rng(41)
+    P, W, T = 7, 9, 4
+    for event_order in (False, True):
+        theta_a, theta_b = np.linspace(-1, 1, P), np.linspace(-1, 1, P)
+        avg_a, avg_b = theta_a.copy(), theta_b.copy()
+        sa = [np.zeros(P), np.zeros(P)]
+        sb = [np.zeros(P), np.zeros(P)]
+        acc, state = np.full(P, np.nan), oracle.new_server_state()
+        seen = 0
+        prev = None
+        for t in range(T):
+            arrival = rng.lognormal(0.0, 0.5, W).astype(np.float32)
+            arrival[rng.integers(0, W)] = np.inf
+            tags = np.where(rng.random(W) < 0.2, t - 1, t).astype(np.int32)
+            grad = rng.standard_normal((W, P)).astype(np.float32)
+            deadline = float(np.float32(np.sort(arrival)[W // 2]))  # somewhere in the middle: an arrival exactly at it is kept
+            opt = oracle.Opt(kind=kind, lr=0.05, decay=0.9, momentum=0.9, eps=1.0)
+            rc_b, mask, order, n = oracle.step_deadline(grad, P, arrival, tags, t, deadline, 1, theta_b, sb[0], sb[1], opt)
+            ids = [int(w) for w in np.argsort(arrival, kind="stable")]
+            early = [w for w in ids if np.isfinite(arrival[w]) and arrival[w] <= np.float32(deadline)]
+            late = [w for w in ids if np.isfinite(arrival[w]) and not arrival[w] <= np.float32(deadline)]
+            outcomes = {}
+            deliveries = early + ([] if event_order else late)
+            if prev is not None:
+                assert oracle.accumulate_arrival_deadline(prev, t - 1, 0.0, t, deadline, acc, state) == 0  # straggler of t - 1
+                seen += 1
+            for w in deliveries:
+                outcomes[w] = oracle.accumulate_arrival_deadline(grad[w], int(tags[w]), float(arrival[w]), t, deadline, acc, state)
+                seen += 1
+            theta_t = theta_a.copy()
+            rc_a, outcome = oracle.accumulate_close(t, 1, acc, state, theta_a, sa[0], sa[1], opt, avg_a, 0.9)
+            assert rc_a == rc_b
+            if rc_b == oracle.OK:
+                assert outcome == 2 and state.tolist() == [0, seen, t + 1]
+                assert sorted(w for w, o in outcomes.items() if o == 1) == sorted(order.tolist()) and n == len(order)
+                assert np.array_equal(avg_a, 0.9 * avg_b + (1.0 - 0.9) * theta_t)
+                avg_b = avg_a.copy()
+            else:
+                assert outcome == 0 and np.array_equal(theta_a, theta_t) and state[2] == t
+                state[0] = 0  # the test moves on: forget the incomplete iteration
+                state[2] = t + 1
+            if event_order:
+                for w in late:
+                    assert oracle.accumulate_arrival_deadline(grad[w], int(tags[w]), float(arrival[w]), t, deadline, acc, state) == 0
+                    seen += 1
+            # closing again, or closing an older iteration, does nothing
+            before = theta_a.copy()
+            assert oracle.accumulate_close(t, 1, acc, state, theta_a, sa[0], sa[1], opt) == (oracle.OK, 0)
+            assert np.array_equal(theta_a, before)
+            assert np.array_equal(theta_a, theta_b) and np.array_equal(sa[0], sb[0]) and np.array_equal(sa[1], sb[1])
+            prev = grad[0].copy()
+
+
+def test_arrival_server_with_deadline_needs_n_min_and_divides_by_the_set():
+    P = 3
+    rows = np.array([[1, 2, 4], [3, 6, 12], [100, 100, 100]], np.float32)
+    acc, state = np.zeros(P), oracle.new_server_state()
+    theta = np.zeros(P)
+    opt = oracle.Opt(kind=oracle.SGD, lr=1.0)
+    assert oracle.accumulate_arrival_deadline(rows[0], 5, 1.0, 5, 2.0, acc, state) == 1
+    assert oracle.accumulate_close(5, 2, acc, state, theta, None, None, opt) == (oracle.INSUFFICIENT, 0)
+    assert theta.tolist() == [0, 0, 0] and state.tolist() == [1, 1, 0]  # the server may keep listening
+    assert oracle.accumulate_arrival_deadline(rows[1], 5, 2.0, 5, 2.0, acc, state) == 1  # exactly at the deadline: kept
+    assert oracle.accumulate_arrival_deadline(rows[2], 5, 2.5, 5, 2.0, acc, state) == 0  # after it: dropped
+    assert oracle.accumulate_arrival_deadline(rows[2], 5, float("nan"), 5, 2.0, acc, state) == 0
+    assert oracle.accumulate_close(5, 2, acc, state, theta, None, None, opt) == (oracle.OK, 2)
+    assert theta.tolist() == [-2.0, -4.0, -8.0] and state.tolist() == [0, 4, 6]  # mean of two, not of three or four
