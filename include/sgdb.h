@@ -19,7 +19,8 @@
  *     Calls only enqueue work; they never synchronise the stream, except the
  *     `_host` entry point, which says so.
  *   - Nothing is allocated by the library; the only memory it touches is what the
- *     caller passes.
+ *     caller passes -- except sgdb_step_host_static, which works in a fixed array that is
+ *     part of the library image.
  *   - Arguments that can be checked on the host (null pointers, N < 1, b < 0,
  *     N + b > SGDB_MAX_WORKERS, P < 0, ld < P, misaligned base pointers, unknown
  *     enum values, non-finite hyper-parameters) make the call return
@@ -227,14 +228,42 @@ sgdb_status_t sgdb_step_deadline(const void *d_grad, sgdb_dtype_t dt, int64_t P,
  * in one launch driven by a table in DEVICE memory (d_segments [S]).  One
  * selection serves all tensors, as one server iteration does in Algorithm 4.
  * S <= SGDB_MAX_SEGMENTS, otherwise SGDB_ERR_UNSUPPORTED.  The table cannot be
- * inspected from the host: a segment with a null theta or grad pointer, or without a
- * state pointer its rule needs, is skipped by the kernel and d_info[1] then reads
- * SGDB_ERR_INVALID_ARG (the other segments are still updated).
+ * inspected from the host: a segment with a null theta or grad pointer, without a
+ * state pointer its rule needs, with a pointer that is not aligned to its element type or
+ * with ld < len is skipped by the kernel and d_info[1] then reads SGDB_ERR_INVALID_ARG (the
+ * other segments are still updated).
  */
 sgdb_status_t sgdb_step_segmented(const sgdb_segment_t *d_segments, int32_t S, sgdb_dtype_t dt,
                                   const float *d_arrival, const int32_t *d_tags, int32_t t,
                                   int32_t N, int32_t b, const sgdb_opt_t *opt, uint8_t *d_mask,
                                   int32_t *d_order, int32_t *d_info, void *stream);
+
+/*
+ * sgdb_step_segmented_ema -- sgdb_step_segmented that also keeps the parameter average of
+ * Algorithm 4's last line (which the algorithm runs for every variable) for each tensor, in
+ * the same launch, from the parameters as they were before the update (see sgdb_step_ema).
+ *   d_ema [S]  DEVICE array of device pointers, entry i = fp32 [len_i] average of tensor i
+ *              (element-aligned; 16-byte aligned is faster); a NULL entry: no average for
+ *              that tensor.  alpha in [0, 1].
+ *
+ * sgdb_step_segmented_deadline -- sgdb_step_segmented with the time-out rule of
+ * sgdb_step_deadline (Section 6): W workers, every gradient tagged t that arrived by
+ * `deadline` is used, at least n_min of them; d_order has W entries, d_info = {n, status}.
+ *
+ * In all three calls an entry of the table whose pointers are missing or not aligned to
+ * their element type, or whose ld is smaller than its len, is skipped and reported as
+ * SGDB_ERR_INVALID_ARG in d_info[1].
+ */
+sgdb_status_t sgdb_step_segmented_ema(const sgdb_segment_t *d_segments, float *const *d_ema, float alpha,
+                                      int32_t S, sgdb_dtype_t dt, const float *d_arrival,
+                                      const int32_t *d_tags, int32_t t, int32_t N, int32_t b,
+                                      const sgdb_opt_t *opt, uint8_t *d_mask, int32_t *d_order,
+                                      int32_t *d_info, void *stream);
+sgdb_status_t sgdb_step_segmented_deadline(const sgdb_segment_t *d_segments, int32_t S, sgdb_dtype_t dt,
+                                           const float *d_arrival, const int32_t *d_tags, int32_t t,
+                                           int32_t W, float deadline, int32_t n_min, const sgdb_opt_t *opt,
+                                           uint8_t *d_mask, int32_t *d_order, int32_t *d_info,
+                                           void *stream);
 
 /*
  * sgdb_select_grouped, sgdb_step_grouped -- two-level aggregation: the gradients of workers
@@ -277,7 +306,8 @@ sgdb_status_t sgdb_step_grouped(const void *d_grad, sgdb_dtype_t dt, int64_t P, 
  * gradient per call, in the order the gradients reach the server.
  *
  *   d_row     [P] of type dt   the arriving gradient; any element-aligned address (a row of
- *                              a matrix with an odd pitch is fine), 16-byte aligned is faster
+ *                              a matrix with an odd pitch is fine; an address that is not a
+ *                              multiple of the element size is refused), 16-byte aligned is faster
  *   row_tag, t                 its tag and the server's iteration
  *   d_acc     [P] fp32         running sum, owned by the caller; needs no clearing:
  *                              the first accepted arrival of an iteration overwrites it
@@ -309,6 +339,31 @@ sgdb_status_t sgdb_accumulate_arrival_ema(const void *d_row, sgdb_dtype_t dt, in
                                           int32_t *d_counter, float *d_theta, float *d_state0,
                                           float *d_state1, const sgdb_opt_t *opt, float *d_ema,
                                           float alpha, int32_t *d_info, void *stream);
+
+/*
+ * sgdb_accumulate_arrival_deadline, sgdb_accumulate_close -- the time-out rule (Section 6, see
+ * sgdb_select_deadline) with one gradient per call.  The server listens until `deadline`:
+ * a gradient joins the running sum iff row_tag == t, iteration t is still open and
+ * row_arrival is finite and <= deadline; there is no upper count.  d_info = {0 dropped |
+ * 1 accumulated, gradients in the set after this call}.  d_row, d_acc, d_counter as in
+ * sgdb_accumulate_arrival; row_arrival and deadline are host values (NaN deadline is refused).
+ *
+ * sgdb_accumulate_close says that the deadline of iteration t has passed.  With at least
+ * n_min (>= 1) gradients in the set, theta moves by their mean (the divisor is the number
+ * in the set), the set is emptied and iteration t + 1 opens: d_info = {2, that number}.
+ * With fewer, or when t is already closed, nothing changes: d_info = {0, gradients in the
+ * set}; the caller may keep delivering and close again later.  d_ema may be NULL; otherwise
+ * the parameter average of Algorithm 4's last line moves with the update, as in sgdb_step_ema.
+ * Delivered in arrival sequence, the result has the bits of sgdb_step_deadline.
+ */
+sgdb_status_t sgdb_accumulate_arrival_deadline(const void *d_row, sgdb_dtype_t dt, int32_t row_tag,
+                                               float row_arrival, int32_t t, float deadline, int64_t P,
+                                               float *d_acc, int32_t *d_counter, int32_t *d_info,
+                                               void *stream);
+sgdb_status_t sgdb_accumulate_close(int32_t t, int32_t n_min, int64_t P, const float *d_acc,
+                                    int32_t *d_counter, float *d_theta, float *d_state0, float *d_state1,
+                                    const sgdb_opt_t *opt, float *d_ema, float alpha, int32_t *d_info,
+                                    void *stream);
 
 /*
  * sgdb_step_host -- sgdb_step for a server whose gradients arrive in HOST memory

@@ -16,7 +16,7 @@ __all__ = ["binding", "workload", "build"]
 _BINDING_NAMES = (
     "sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented", "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate",
     "sgdb_accumulate_arrival", "sgdb_accumulate_arrival_ema", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
-    "sgdb_select_grouped", "sgdb_step_grouped", "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version", "Opt", "SgdbError",
+    "sgdb_select_grouped", "sgdb_step_grouped", "sgdb_step_segmented_ema", "sgdb_step_segmented_deadline", "sgdb_accumulate_arrival_deadline", "sgdb_accumulate_close", "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version", "Opt", "SgdbError",
 )
 
 

@@ -26,7 +26,8 @@ _KINDS = {"sgd": SGDB_SGD, "momentum": SGDB_MOMENTUM, "rmsprop": SGDB_RMSPROP, "
 EXPORTS = (
     "sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented",
     "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_accumulate_arrival_ema", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
-    "sgdb_select_grouped", "sgdb_step_grouped", "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version",
+    "sgdb_select_grouped", "sgdb_step_grouped", "sgdb_step_segmented_ema", "sgdb_step_segmented_deadline",
+    "sgdb_accumulate_arrival_deadline", "sgdb_accumulate_close", "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version",
 )
 SGDB_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -94,6 +95,12 @@ def _load():
         "sgdb_ema": (i32, [vp, vp, i64, ctypes.c_float, vp, vp]),
         "sgdb_learning_rate": (ctypes.c_double, [ctypes.c_double, ctypes.c_double, i64, i64, ctypes.c_double]),
         "sgdb_step_segmented": (i32, [vp, i32, i32, vp, vp, i32, i32, i32, ctypes.POINTER(_COpt), vp, vp, vp, vp]),
+        "sgdb_step_segmented_ema": (i32, [vp, vp, ctypes.c_float, i32, i32, vp, vp, i32, i32, i32, ctypes.POINTER(_COpt),
+                                          vp, vp, vp, vp]),
+        "sgdb_step_segmented_deadline": (i32, [vp, i32, i32, vp, vp, i32, i32, ctypes.c_float, i32, ctypes.POINTER(_COpt),
+                                               vp, vp, vp, vp]),
+        "sgdb_accumulate_arrival_deadline": (i32, [vp, i32, i32, ctypes.c_float, i32, ctypes.c_float, i64, vp, vp, vp, vp]),
+        "sgdb_accumulate_close": (i32, [i32, i32, i64, vp, vp, vp, vp, vp, ctypes.POINTER(_COpt), vp, ctypes.c_float, vp, vp]),
         "sgdb_select_grouped": (i32, [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]),
         "sgdb_step_grouped": (i32, [vp, i32, i64, i64, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt),
                                     vp, vp, vp, vp, vp]),
@@ -283,6 +290,59 @@ def sgdb_step_segmented(table, S: int, grad_dtype, arrival, tags, t: int, N: int
                                     t, N, b, ctypes.byref(c), _dev(mask, torch.uint8, "mask"),
                                     _dev(order, torch.int32, "order"), _dev(info, torch.int32, "info"),
                                     _stream(stream)), "sgdb_step_segmented")
+
+
+def make_pointer_table(tensors, device) -> torch.Tensor:
+    """Device array of device pointers (int64 CUDA tensor) from a list of CUDA tensors; None -> NULL.
+    The caller keeps the listed tensors alive."""
+    return torch.tensor([0 if x is None else _dev(x, torch.float32, "tensor") for x in tensors], dtype=torch.int64).to(device)
+
+
+def sgdb_step_segmented_ema(table, ema_table, alpha: float, S: int, grad_dtype, arrival, tags, t: int, N: int, b: int,
+                            opt: Opt, mask, order, info, stream=None) -> None:
+    """sgdb_step_segmented plus the per-tensor parameter averages (ema_table from make_pointer_table)."""
+    dt = SGDB_BF16 if grad_dtype == torch.bfloat16 else SGDB_F32
+    c = opt._c()
+    _check(_lib.sgdb_step_segmented_ema(_dev(table, torch.uint8, "segment table"), _dev(ema_table, torch.int64, "ema table"),
+                                        alpha, S, dt, _dev(arrival, torch.float32, "arrival"),
+                                        _dev(tags, torch.int32, "tags"), t, N, b, ctypes.byref(c),
+                                        _dev(mask, torch.uint8, "mask"), _dev(order, torch.int32, "order"),
+                                        _dev(info, torch.int32, "info"), _stream(stream)), "sgdb_step_segmented_ema")
+
+
+def sgdb_step_segmented_deadline(table, S: int, grad_dtype, arrival, tags, t: int, deadline: float, n_min: int, opt: Opt,
+                                 mask, order, info, stream=None) -> None:
+    """sgdb_step_segmented with the time-out rule; order has W entries, info = {n, status}."""
+    dt = SGDB_BF16 if grad_dtype == torch.bfloat16 else SGDB_F32
+    W = arrival.numel()
+    c = opt._c()
+    _check(_lib.sgdb_step_segmented_deadline(_dev(table, torch.uint8, "segment table"), S, dt,
+                                             _dev(arrival, torch.float32, "arrival"), _dev(tags, torch.int32, "tags"),
+                                             t, W, deadline, n_min, ctypes.byref(c), _dev(mask, torch.uint8, "mask"),
+                                             _dev(order, torch.int32, "order"), _dev(info, torch.int32, "info"),
+                                             _stream(stream)), "sgdb_step_segmented_deadline")
+
+
+def sgdb_accumulate_arrival_deadline(row, row_tag: int, row_arrival: float, t: int, deadline: float, acc, counter, info,
+                                     P: int | None = None, stream=None) -> None:
+    """Time-out rule, one arriving gradient: joins the running sum iff tagged t, t open and arrived by the deadline."""
+    P = acc.numel() if P is None else P
+    _check(_lib.sgdb_accumulate_arrival_deadline(_dev(row, None, "row"), _grad_dtype(row), row_tag, row_arrival, t,
+                                                 deadline, P, _dev(acc, torch.float32, "acc"),
+                                                 _dev(counter, torch.int32, "counter"), _dev(info, torch.int32, "info"),
+                                                 _stream(stream)), "sgdb_accumulate_arrival_deadline")
+
+
+def sgdb_accumulate_close(t: int, n_min: int, acc, counter, theta, state0, state1, opt: Opt, info, ema=None,
+                          alpha: float = 0.0, P: int | None = None, stream=None) -> None:
+    """The deadline of iteration t has passed: update from the mean of the set if it holds at least n_min gradients."""
+    P = theta.numel() if P is None else P
+    c = opt._c()
+    _check(_lib.sgdb_accumulate_close(t, n_min, P, _dev(acc, torch.float32, "acc"), _dev(counter, torch.int32, "counter"),
+                                      _dev(theta, torch.float32, "theta"), _dev(state0, torch.float32, "state0"),
+                                      _dev(state1, torch.float32, "state1"), ctypes.byref(c),
+                                      _dev(ema, torch.float32, "ema"), alpha, _dev(info, torch.int32, "info"),
+                                      _stream(stream)), "sgdb_accumulate_close")
 
 
 def sgdb_select_grouped(arrival, tags, group, t: int, M: int, N: int, mask, group_order, order, info, stream=None) -> None:

@@ -287,6 +287,23 @@ sgdb_status_t check_flat(const void* grad, int dt, int64_t P, int64_t ld, int32_
   return SGDB_OK;
 }
 
+// Launch with programmatic stream serialization, like every kernel that works on the server state.
+template <typename Kernel, typename Params>
+sgdb_status_t launch_on_server_state(Kernel kernel, unsigned grid, const Params& p, cudaStream_t s) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = SGDB_PDL ? 1 : 0;
+  (void)cudaLaunchKernelEx(&cfg, kernel, p);
+  return launch_status();
+}
+
 }  // namespace
 
 // ====================================================================== C ABI
@@ -444,11 +461,12 @@ sgdb_status_t sgdb_step_deadline(const void* d_grad, sgdb_dtype_t dt, int64_t P,
   return launch_stream(dt, ep, p, static_cast<cudaStream_t>(stream));
 }
 
-sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, sgdb_dtype_t dt,
-                                  const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t N,
-                                  int32_t b, const sgdb_opt_t* opt, uint8_t* d_mask, int32_t* d_order,
-                                  int32_t* d_info, void* stream) {
-  sgdb_status_t st = check_selection_args(d_arrival, d_tags, N, b, d_mask, d_order, d_info);
+// The multi-tensor step in its three forms: first-N rule, first-N rule with per-tensor averages, time-out rule.
+static sgdb_status_t step_segmented(const sgdb_segment_t* d_segments, int32_t S, sgdb_dtype_t dt,
+                                    const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t N, int32_t b,
+                                    bool keep_all, float deadline, const sgdb_opt_t* opt, float* const* d_ema,
+                                    float alpha, uint8_t* d_mask, int32_t* d_order, int32_t* d_info, void* stream) {
+  sgdb_status_t st = check_selection_args(d_arrival, d_tags, keep_all ? N + b : N, keep_all ? 0 : b, d_mask, d_order, d_info);
   if (st != SGDB_OK) return st;
   if (d_segments == nullptr || S < 0 || !dtype_ok(dt)) return SGDB_ERR_INVALID_ARG;
   if (S > SGDB_MAX_SEGMENTS) return SGDB_ERR_UNSUPPORTED;
@@ -460,14 +478,52 @@ sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, s
   st = prepare_rule(opt, &dummy, &dummy, &h, &ep);
   if (st != SGDB_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (S == 0) return launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
+  const int32_t W = N + b;
+  if (S == 0) {
+    if (!keep_all) return launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
+    return sgdb_select_deadline(d_arrival, d_tags, t, W, deadline, N, d_mask, d_order, d_info, stream);
+  }
   StreamParams p{};
   p.table = d_segments;
   p.S = S;
-  p.N = N;
-  set_in_kernel_selection(&p, d_arrival, d_tags, t, N + b, d_mask, d_order, d_info);
+  p.N = N;  // with the time-out rule: the fewest gradients accepted
+  set_in_kernel_selection(&p, d_arrival, d_tags, t, W, d_mask, d_order, d_info);
+  if (keep_all) {
+    p.deadline = deadline;
+    p.keep_all = true;
+    p.order_cap = W;
+  }
+  p.ema_table = d_ema;
+  p.ema_alpha = alpha;
+  p.ema_one_minus_alpha = static_cast<float>(1.0 - static_cast<double>(alpha));
   p.h = h;
   return launch_stream(dt, ep, p, s);
+}
+
+sgdb_status_t sgdb_step_segmented(const sgdb_segment_t* d_segments, int32_t S, sgdb_dtype_t dt,
+                                  const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t N,
+                                  int32_t b, const sgdb_opt_t* opt, uint8_t* d_mask, int32_t* d_order,
+                                  int32_t* d_info, void* stream) {
+  return step_segmented(d_segments, S, dt, d_arrival, d_tags, t, N, b, false, kNoDeadline, opt, nullptr, 0.0f, d_mask,
+                        d_order, d_info, stream);
+}
+
+sgdb_status_t sgdb_step_segmented_ema(const sgdb_segment_t* d_segments, float* const* d_ema, float alpha, int32_t S,
+                                      sgdb_dtype_t dt, const float* d_arrival, const int32_t* d_tags, int32_t t,
+                                      int32_t N, int32_t b, const sgdb_opt_t* opt, uint8_t* d_mask, int32_t* d_order,
+                                      int32_t* d_info, void* stream) {
+  if (d_ema == nullptr || !(alpha >= 0.0f && alpha <= 1.0f)) return SGDB_ERR_INVALID_ARG;
+  return step_segmented(d_segments, S, dt, d_arrival, d_tags, t, N, b, false, kNoDeadline, opt, d_ema, alpha, d_mask,
+                        d_order, d_info, stream);
+}
+
+sgdb_status_t sgdb_step_segmented_deadline(const sgdb_segment_t* d_segments, int32_t S, sgdb_dtype_t dt,
+                                           const float* d_arrival, const int32_t* d_tags, int32_t t, int32_t W,
+                                           float deadline, int32_t n_min, const sgdb_opt_t* opt, uint8_t* d_mask,
+                                           int32_t* d_order, int32_t* d_info, void* stream) {
+  if (W < 1 || n_min < 1 || n_min > W || std::isnan(deadline)) return SGDB_ERR_INVALID_ARG;
+  return step_segmented(d_segments, S, dt, d_arrival, d_tags, t, n_min, W - n_min, true, deadline, opt, nullptr, 0.0f,
+                        d_mask, d_order, d_info, stream);
 }
 
 static sgdb_status_t check_grouped_args(const void* arrival, const void* tags, const void* group, int32_t W, int32_t M,
@@ -538,7 +594,7 @@ static sgdb_status_t arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag
   st = device_info(&dev);
   if (st != SGDB_OK) return st;
   ArrivalParams p{d_row, row_tag, t, N, P, d_acc, d_counter, d_theta, d_state0, d_state1, d_info,
-                  d_ema, alpha, static_cast<float>(1.0 - static_cast<double>(alpha)), g_arrival_resident_bytes / 4, h};
+                  d_ema, alpha, static_cast<float>(1.0 - static_cast<double>(alpha)), g_arrival_resident_bytes / 4, 1, h};
   const int V = dt == SGDB_BF16 ? 8 : 4;
   const long long chunks = (P + V - 1) / V;
   long long grid = (chunks + 4 * 256 - 1) / (4 * 256);  // at least 4 chunks per thread
@@ -547,31 +603,19 @@ static sgdb_status_t arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag
   if (row_tag != t || grid < 1) grid = 1;  // a wrongly tagged gradient only updates the bookkeeping
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const unsigned g = static_cast<unsigned>(grid);
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(g);
-  cfg.blockDim = dim3(256);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = SGDB_PDL ? 1 : 0;
-#define SGDB_ARRIVAL_CASE(EPV)                                                               \
-  case EPV:                                                                                  \
-    if (dt == SGDB_BF16) (void)cudaLaunchKernelEx(&cfg, accumulate_arrival_kernel<BF16, EPV>, p); \
-    else (void)cudaLaunchKernelEx(&cfg, accumulate_arrival_kernel<float, EPV>, p);                \
-    break;
+#define SGDB_ARRIVAL_CASE(EPV)                                                                               \
+  case EPV:                                                                                                  \
+    return dt == SGDB_BF16 ? launch_on_server_state(accumulate_arrival_kernel<BF16, EPV>, g, p, s)           \
+                           : launch_on_server_state(accumulate_arrival_kernel<float, EPV>, g, p, s);
   switch (ep) {
     SGDB_ARRIVAL_CASE(EP_SGD)
     SGDB_ARRIVAL_CASE(EP_MOMENTUM)
     SGDB_ARRIVAL_CASE(EP_RMSPROP)
     SGDB_ARRIVAL_CASE(EP_ADAM)
     SGDB_ARRIVAL_CASE(EP_ADAGRAD)
-    default: return SGDB_ERR_INVALID_ARG;
   }
 #undef SGDB_ARRIVAL_CASE
-  return launch_status();
+  return SGDB_ERR_INVALID_ARG;
 }
 
 sgdb_status_t sgdb_accumulate_arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag, int32_t t,
@@ -590,6 +634,65 @@ sgdb_status_t sgdb_accumulate_arrival_ema(const void* d_row, sgdb_dtype_t dt, in
   if (d_ema == nullptr || !(alpha >= 0.0f && alpha <= 1.0f)) return SGDB_ERR_INVALID_ARG;
   return arrival(d_row, dt, row_tag, t, N, P, d_acc, d_counter, d_theta, d_state0, d_state1, opt, d_ema, alpha, d_info,
                  stream);
+}
+
+sgdb_status_t sgdb_accumulate_arrival_deadline(const void* d_row, sgdb_dtype_t dt, int32_t row_tag, float row_arrival,
+                                               int32_t t, float deadline, int64_t P, float* d_acc, int32_t* d_counter,
+                                               int32_t* d_info, void* stream) {
+  if (d_row == nullptr || d_acc == nullptr || d_counter == nullptr || d_info == nullptr) return SGDB_ERR_INVALID_ARG;
+  if (!dtype_ok(dt) || P < 0 || std::isnan(deadline)) return SGDB_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_row) % dtype_size(dt) != 0 || !is_aligned16(d_acc)) return SGDB_ERR_INVALID_ARG;
+  const DeviceInfo* dev = nullptr;
+  sgdb_status_t st = device_info(&dev);
+  if (st != SGDB_OK) return st;
+  const bool in_time = std::isfinite(row_arrival) && row_arrival <= deadline;
+  // no upper count with the time-out rule: N is out of reach, so this launch never completes a set
+  ArrivalParams p{d_row, row_tag, t, std::numeric_limits<int32_t>::max(), P, d_acc, d_counter, nullptr, nullptr, nullptr,
+                  d_info, nullptr, 0.0f, 1.0f, g_arrival_resident_bytes / 4, in_time ? 1 : 0, Hyper{}};
+  const int V = dt == SGDB_BF16 ? 8 : 4;
+  const long long chunks = (P + V - 1) / V;
+  long long grid = (chunks + 4 * 256 - 1) / (4 * 256);
+  const long long cap = static_cast<long long>(dev->sms) * g_arrival_blocks_per_sm;
+  if (grid > cap) grid = cap;
+  if (row_tag != t || !in_time || grid < 1) grid = 1;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dt == SGDB_BF16) return launch_on_server_state(accumulate_arrival_kernel<BF16, EP_SGD>, static_cast<unsigned>(grid), p, s);
+  return launch_on_server_state(accumulate_arrival_kernel<float, EP_SGD>, static_cast<unsigned>(grid), p, s);
+}
+
+sgdb_status_t sgdb_accumulate_close(int32_t t, int32_t n_min, int64_t P, const float* d_acc, int32_t* d_counter,
+                                    float* d_theta, float* d_state0, float* d_state1, const sgdb_opt_t* opt,
+                                    float* d_ema, float alpha, int32_t* d_info, void* stream) {
+  if (d_acc == nullptr || d_counter == nullptr || d_theta == nullptr || d_info == nullptr) return SGDB_ERR_INVALID_ARG;
+  if (n_min < 1 || P < 0) return SGDB_ERR_INVALID_ARG;
+  if (d_ema != nullptr && !(alpha >= 0.0f && alpha <= 1.0f)) return SGDB_ERR_INVALID_ARG;
+  if (!is_aligned16(d_acc) || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1) ||
+      !is_aligned16(d_ema))
+    return SGDB_ERR_INVALID_ARG;
+  Hyper h;
+  int ep = 0;
+  sgdb_status_t st = prepare_rule(opt, d_state0, d_state1, &h, &ep);
+  if (st != SGDB_OK) return st;
+  const DeviceInfo* dev = nullptr;
+  st = device_info(&dev);
+  if (st != SGDB_OK) return st;
+  CloseParams p{t, n_min, P, d_acc, d_counter, d_theta, d_state0, d_state1, d_info, d_ema, alpha,
+                static_cast<float>(1.0 - static_cast<double>(alpha)), h};
+  const long long chunks = (P + 3) / 4;
+  long long grid = (chunks + 255) / 256;
+  const long long cap = static_cast<long long>(dev->sms) * 8;
+  if (grid > cap) grid = cap;
+  if (grid < 1) grid = 1;
+  const unsigned g = static_cast<unsigned>(grid);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  switch (ep) {
+    case EP_SGD: return launch_on_server_state(close_iteration_kernel<EP_SGD>, g, p, s);
+    case EP_MOMENTUM: return launch_on_server_state(close_iteration_kernel<EP_MOMENTUM>, g, p, s);
+    case EP_RMSPROP: return launch_on_server_state(close_iteration_kernel<EP_RMSPROP>, g, p, s);
+    case EP_ADAM: return launch_on_server_state(close_iteration_kernel<EP_ADAM>, g, p, s);
+    case EP_ADAGRAD: return launch_on_server_state(close_iteration_kernel<EP_ADAGRAD>, g, p, s);
+  }
+  return SGDB_ERR_INVALID_ARG;
 }
 
 // Workspace layout of sgdb_step_host: arrival[W] f32 | tags[W] i32 | order[N] i32 | info[2] i32 |

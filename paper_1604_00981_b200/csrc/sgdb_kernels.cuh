@@ -317,9 +317,11 @@ struct StreamParams {
   const int32_t* group;
   int32_t M;
   int32_t* group_order_out;
-  // Optional (flat case): exponential moving average of the parameters, updated in the
-  // same pass from the value theta had BEFORE this step's update.
+  // Optional: exponential moving average of the parameters, updated in the same pass from the
+  // value theta had BEFORE this step's update.  Flat case: `ema`; with a segment table:
+  // `ema_table` [S] device pointers, one per tensor (a null entry: that tensor keeps no average).
   float* ema;
+  float* const* ema_table;
   float ema_alpha, ema_one_minus_alpha;
   Hyper h;
 };
@@ -338,12 +340,28 @@ struct TileDesc {
   bool bad;       // a pointer this rule needs is null in the segment table: the tile is skipped
 };
 
+// A table entry the kernel may use: the pointers its rule needs are there and aligned to their
+// element type, and the rows do not overlap (ld >= len).  The table lives in device memory, so the
+// host cannot check it; an entry that fails is left alone and reported instead of being dereferenced.
+template <typename GT, int EP>
+__device__ __forceinline__ bool segment_usable(const sgdb_segment_t& seg, const float* ema) {
+  using Rule = RuleTraits<EP>;
+  if (seg.theta == nullptr || seg.grad == nullptr || (Rule::kState0 && seg.state0 == nullptr) ||
+      (Rule::kState1 && seg.state1 == nullptr))
+    return false;
+  const uintptr_t fp32_ptrs = reinterpret_cast<uintptr_t>(seg.theta) | reinterpret_cast<uintptr_t>(seg.state0) |
+                              reinterpret_cast<uintptr_t>(seg.state1) | reinterpret_cast<uintptr_t>(ema);
+  if ((fp32_ptrs & 3u) != 0 || (reinterpret_cast<uintptr_t>(seg.grad) & (sizeof(GT) - 1)) != 0) return false;
+  return seg.ld >= seg.len;
+}
+
 template <typename GT, int TILE, int EP>
 __device__ __forceinline__ TileDesc<GT> locate_tile(const StreamParams& p, const int* prefix_s,
                                                     int tile) {
   constexpr int V = GradTraits<GT>::kVec;
   sgdb_segment_t seg;
   long long col0;
+  float* ema = p.ema;
   if (p.table == nullptr) {
     seg = p.flat;
     col0 = static_cast<long long>(tile) * TILE;
@@ -355,6 +373,7 @@ __device__ __forceinline__ TileDesc<GT> locate_tile(const StreamParams& p, const
     }
     seg = p.table[lo];
     col0 = static_cast<long long>(tile - prefix_s[lo]) * TILE;
+    ema = p.ema_table != nullptr ? p.ema_table[lo] : nullptr;
   }
   TileDesc<GT> td;
   td.grad = static_cast<const GT*>(seg.grad) + col0;
@@ -368,14 +387,10 @@ __device__ __forceinline__ TileDesc<GT> locate_tile(const StreamParams& p, const
                        (((seg.ld * static_cast<long long>(sizeof(GT))) & 15) == 0);
   td.bulk_cols = bulk_ok ? (td.ncols / V) * V : 0;
   td.bad = false;
-  td.ema = (p.ema != nullptr && p.table == nullptr) ? p.ema + col0 : nullptr;
+  td.ema = ema != nullptr ? ema + col0 : nullptr;
   td.vec_ok = (((reinterpret_cast<uintptr_t>(seg.theta) | reinterpret_cast<uintptr_t>(seg.state0) |
-                 reinterpret_cast<uintptr_t>(seg.state1) | reinterpret_cast<uintptr_t>(p.ema)) & 15u) == 0);
-  // The table lives in device memory, so the host cannot check it: a segment without a
-  // pointer its rule needs is left alone (and reported) instead of being dereferenced.
-  using Rule = RuleTraits<EP>;
-  if (seg.theta == nullptr || seg.grad == nullptr || (Rule::kState0 && seg.state0 == nullptr) ||
-      (Rule::kState1 && seg.state1 == nullptr)) {
+                 reinterpret_cast<uintptr_t>(seg.state1) | reinterpret_cast<uintptr_t>(ema)) & 15u) == 0);
+  if (p.table != nullptr && !segment_usable<GT, EP>(seg, ema)) {
     td.bad = true;
     td.ncols = 0;
     td.bulk_cols = 0;
@@ -442,15 +457,13 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
   }
   if (p.table != nullptr) {
     // tiles per segment, then an inclusive scan: prefix_s[i] = tiles in segments < i
-    // The same pass looks for entries that lack a pointer this rule needs (the host cannot
-    // see the table); their tiles are skipped below and block 0 reports them once.
+    // The same pass looks for entries the kernel must not use (a missing or misaligned pointer,
+    // rows that overlap); their tiles are skipped below and block 0 reports them once.
     int incomplete = 0;
     for (int i = tid; i < p.S; i += NT + 32) {
       const sgdb_segment_t seg = p.table[i];
       prefix_s[i + 1] = seg.len > 0 ? static_cast<int>((seg.len + TILE - 1) / TILE) : 0;
-      if (seg.len > 0 && (seg.theta == nullptr || seg.grad == nullptr || (Rule::kState0 && seg.state0 == nullptr) ||
-                          (Rule::kState1 && seg.state1 == nullptr)))
-        incomplete = 1;
+      if (seg.len > 0 && !segment_usable<GT, EP>(seg, p.ema_table != nullptr ? p.ema_table[i] : nullptr)) incomplete = 1;
     }
     if (tid == 0) prefix_s[0] = 0;
     incomplete = __syncthreads_or(incomplete);
@@ -786,6 +799,7 @@ struct ArrivalParams {
   float* ema;     // optional: average of the parameters, moved when the update fires
   float ema_alpha, ema_one_minus_alpha;
   long long acc_resident;  // leading elements of acc that are asked to stay in L2 between launches
+  int32_t admissible;      // 0: the host already knows this gradient is dropped (it arrived after the deadline)
   Hyper h;
 };
 
@@ -816,7 +830,7 @@ __global__ void __launch_bounds__(256, 4) accumulate_arrival_kernel(const Arriva
   }
   __syncthreads();
   const int accepted = s_accepted;
-  const bool admit = (p.row_tag == p.t) && (p.t >= s_open) && (accepted < p.N);
+  const bool admit = p.admissible != 0 && (p.row_tag == p.t) && (p.t >= s_open) && (accepted < p.N);
   const bool first = accepted == 0;          // the set was empty: start the sum from +0
   const bool last = accepted + 1 == p.N;     // this gradient completes the set
 
@@ -931,6 +945,87 @@ __global__ void __launch_bounds__(256, 4) accumulate_arrival_kernel(const Arriva
       }
       p.info[0] = outcome;
       p.info[1] = after;
+    }
+  }
+}
+
+// ====================================================================== closing an iteration
+//
+// Time-out rule, arrival by arrival: the deadline of iteration t has passed.  With at least n_min
+// gradients in the running sum the parameters move by their mean (divisor: the number accepted),
+// the set is emptied and t + 1 opens; otherwise nothing changes.  Same protocol on the server
+// state as the arrival kernel: every block reads it first, the last ticket changes it.
+
+struct CloseParams {
+  int32_t t, n_min;
+  long long P;
+  const float* acc;
+  int32_t* counter;  // [4]
+  float* theta;
+  float* s0;
+  float* s1;
+  int32_t* info;  // [2]: {2 updated | 0 nothing done, gradients in the set}
+  float* ema;     // optional
+  float ema_alpha, ema_one_minus_alpha;
+  Hyper h;
+};
+
+template <int EP>
+__global__ void __launch_bounds__(256, 4) close_iteration_kernel(const CloseParams p) {
+  using Rule = RuleTraits<EP>;
+  __shared__ int s_accepted, s_open;
+#if SGDB_PDL
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
+  if (threadIdx.x == 0) {
+    s_accepted = *reinterpret_cast<volatile int32_t*>(p.counter + 0);
+    s_open = *reinterpret_cast<volatile int32_t*>(p.counter + 3);
+  }
+  __syncthreads();
+  const int accepted = s_accepted;
+  const bool fire = (p.t >= s_open) && (accepted >= p.n_min);
+  if (fire) {
+    const float n_as_float = static_cast<float>(accepted);
+    const uint64_t pol_stream = l2_policy_evict_first();
+    const long long chunks = (p.P + 3) / 4;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long q = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; q < chunks; q += stride) {
+      const long long i = q * 4;
+      const long long rest = p.P - i;
+      const int n = rest < 4 ? static_cast<int>(rest) : 4;
+      const bool vec = n == 4;
+      float a[4], th[4], s0[4], s1[4];
+      load_floats_hint<4>(p.acc + i, vec, n, a, pol_stream);  // last use of the sum
+      load_floats<4>(p.theta + i, vec, n, th);
+      if (Rule::kState0) load_floats<4>(p.s0 + i, vec, n, s0);
+      if (Rule::kState1) load_floats<4>(p.s1 + i, vec, n, s1);
+      if (p.ema != nullptr) {
+        float avg[4];
+        load_floats<4>(p.ema + i, vec, n, avg);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) avg[e] = ema_rule(p.ema_alpha, p.ema_one_minus_alpha, avg[e], th[e]);
+        store_floats<4>(p.ema + i, vec, n, avg);
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) apply_rule<EP>(p.h, __fdiv_rn(a[e], n_as_float), th[e], s0[e], s1[e]);
+      store_floats<4>(p.theta + i, vec, n, th);
+      if (Rule::kState0) store_floats<4>(p.s0 + i, vec, n, s0);
+      if (Rule::kState1) store_floats<4>(p.s1 + i, vec, n, s1);
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned ticket = atomicAdd(reinterpret_cast<unsigned*>(p.counter + 2), 1u);
+    if (ticket == gridDim.x - 1) {
+      p.counter[2] = 0;
+      if (fire) {
+        p.counter[0] = 0;
+        p.counter[3] = p.t + 1;
+      }
+      p.info[0] = fire ? 2 : 0;
+      p.info[1] = accepted;
     }
   }
 }

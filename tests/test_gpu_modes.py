@@ -142,6 +142,18 @@ def test_segmented_edge_cases(sgdb, cuda_device):
                              mask, order, info)
     assert info.cpu().tolist() == [4, sgdb.SGDB_ERR_INVALID_ARG]
     assert (th[0] == -1).all() and (th[1] == 0).all() and (th[2] == -1).all()
+    # entries the kernel must not touch: a pointer that is not aligned to its element, rows that overlap (ld < len)
+    raw = torch.zeros(4 * 5000 + 16, dtype=torch.uint8, device=dev)
+    # (torch refuses misaligned views, so the entries are built by hand)
+    good = [torch.zeros(5000, device=dev) for _ in range(3)]
+    entries = (sgdb.CSegment * 3)()
+    entries[0] = sgdb.CSegment(good[0].data_ptr(), 0, 0, gr[0].data_ptr(), 5000, 5000)
+    entries[1] = sgdb.CSegment(raw.data_ptr() + 2, 0, 0, gr[1].data_ptr(), 5000, 5000)          # theta at a 2-byte offset
+    entries[2] = sgdb.CSegment(good[2].data_ptr(), 0, 0, gr[2].data_ptr(), 4999, 5000)          # ld < len
+    table = torch.frombuffer(bytearray(bytes(entries)), dtype=torch.uint8).to(dev)
+    sgdb.sgdb_step_segmented(table, 3, torch.float32, a_d, t_d, 0, N, 1, gpu_opt(dict(kind="sgd", lr=1.0)), mask, order, info)
+    assert info.cpu().tolist() == [4, sgdb.SGDB_ERR_INVALID_ARG]
+    assert (good[0] == -1).all() and (raw == 0).all() and (good[2] == 0).all()
     # the largest table, every tensor tiny
     S = sgdb.SGDB_MAX_SEGMENTS
     theta = torch.zeros(S * 3, device=dev)
@@ -294,6 +306,26 @@ def test_arrivals_enqueued_back_to_back_without_host_reads(sgdb, cuda_device, ki
         assert x is None or torch.equal(x, y)
     tol = TOL_F32 if dtype == "f32" else TOL_BF16
     assert rel_err(theta[cols_d].cpu().numpy(), th_o) < tol and rel_err(avg[cols_d].cpu().numpy(), avg_o) < tol
+
+
+def test_arriving_row_must_be_element_aligned(sgdb, cuda_device):
+    """A row address that is not a multiple of the element size is refused on the host; nothing is launched."""
+    import ctypes
+
+    dev = cuda_device
+    P = 1000
+    raw = torch.zeros(4 * P + 16, dtype=torch.uint8, device=dev)
+    acc, theta = torch.zeros(P, device=dev), torch.zeros(P, device=dev)
+    counter = torch.zeros(4, dtype=torch.int32, device=dev)
+    info = torch.zeros(2, dtype=torch.int32, device=dev)
+    c = gpu_opt(OPTS["sgd"])._c()
+    for dt, offset, want in ((sgdb.SGDB_F32, 2, sgdb.SGDB_ERR_INVALID_ARG), (sgdb.SGDB_BF16, 1, sgdb.SGDB_ERR_INVALID_ARG),
+                             (sgdb.SGDB_F32, 4, sgdb.SGDB_OK), (sgdb.SGDB_BF16, 2, sgdb.SGDB_OK)):
+        st = sgdb._lib.sgdb_accumulate_arrival(raw.data_ptr() + offset, dt, 0, 0, 4, P, acc.data_ptr(), counter.data_ptr(),
+                                               theta.data_ptr(), 0, 0, ctypes.byref(c), info.data_ptr(), 0)
+        assert st == want
+    torch.cuda.synchronize()
+    assert counter.cpu().tolist()[1] == 2  # only the two aligned rows were seen
 
 
 @pytest.mark.parametrize("kind,dtype", [("sgd", "f32"), ("rmsprop", "bf16")])
