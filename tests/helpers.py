@@ -77,3 +77,23 @@ def to_dev(a: np.ndarray, device) -> torch.Tensor:
 
 def step_inputs(seed: int, t: int, W: int, N: int):
     return wl.arrivals(seed, t, W), wl.tags(seed, t, W, N)
+
+
+def oracle_step_over_column_ranges(grad, P, arrival, tags, t, N, b, theta, s0, s1, opt, threads):
+    """The oracle's step on [W, P] host rows, one unchanged oracle call per contiguous column range, each from its
+    own thread (the oracle itself stays single-threaded; the path is separable by column).  Returns the list of
+    (status, mask, order, n_valid) of the pieces."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    flat = grad.reshape(-1)
+    ld = grad.shape[1]
+    edges = [P * k // threads for k in range(threads + 1)]
+    pieces = [(edges[k], edges[k + 1]) for k in range(threads) if edges[k + 1] > edges[k]]
+
+    def piece(r):
+        c0, c1 = r
+        return oracle.step(flat[c0:], c1 - c0, arrival, tags, t, N, b, theta[c0:c1], None if s0 is None else s0[c0:c1],
+                           None if s1 is None else s1[c0:c1], opt, ld=ld)
+
+    with ThreadPoolExecutor(max_workers=len(pieces)) as pool:
+        return list(pool.map(piece, pieces))

@@ -91,6 +91,48 @@ def test_config1_full_size(sgdb, cuda_device):
     assert torch.equal(theta, th_f) and torch.equal(s0, s0_f) and torch.equal(s1, s1_f)
 
 
+def test_config1_full_size_every_column_against_the_oracle(sgdb, cuda_device):
+    """Two fused steps at P = 23.8 M, W = 100 (N = 96, b = 4), RMSProp, in the launch configuration the benchmark
+    times, and EVERY element of theta and of both state vectors compared with the oracle: the gradient matrix is
+    copied back in column chunks and the oracle runs chunk by chunk (one call per column range and host thread)."""
+    import os
+
+    from helpers import oracle_step_over_column_ranges
+
+    _need_memory(cuda_device, 12)
+    dev, cfg = cuda_device, wl.CONFIGS[1]
+    W, N, P, kind = cfg.W, cfg.N, cfg.P, cfg.opt["kind"]
+    threads = max(1, len(os.sched_getaffinity(0)))
+    scales = wl.worker_scales(cfg.seed, W)
+    theta = wl.theta0(cfg.seed, P, dev)
+    s0, s1 = gpu_state(kind, P, dev)
+    th_o = theta.cpu().numpy().astype(np.float64)
+    s0_o, s1_o = oracle_state(kind, P)
+    mask, order, info = selection_buffers(W, N, dev)
+    chunk = 2_000_000
+    grad = None
+    for t in range(2):
+        grad = wl.grad_matrix(cfg.seed, t, W, P, scales, cfg.grad_dtype, dev, out=grad)
+        arrival, tags = step_inputs(cfg.seed, t, W, N)
+        sgdb.sgdb_step(grad, P, to_dev(arrival, dev), to_dev(tags, dev), t, N, cfg.b, theta, s0, s1,
+                       gpu_opt(cfg.opt, t + 1), mask, order, info)
+        for c0 in range(0, P, chunk):
+            c1 = min(P, c0 + chunk)
+            rows = wl.as_oracle_array(grad[:, c0:c1].contiguous())
+            for rc, mask_o, order_o, n_valid in oracle_step_over_column_ranges(
+                    rows, c1 - c0, arrival, tags, t, N, cfg.b, th_o[c0:c1], s0_o[c0:c1], s1_o[c0:c1],
+                    oracle_opt(cfg.opt, t + 1), threads):
+                assert rc == oracle.OK
+            del rows
+        assert info.cpu().tolist() == [n_valid, 0]
+        assert mask.cpu().numpy().tolist() == mask_o.tolist() and order.cpu().numpy().tolist() == order_o.tolist()
+    got = theta.cpu().numpy()
+    assert rel_err(got, th_o) < TOL_F32
+    assert rel_err(s0.cpu().numpy(), s0_o) < TOL_F32 and rel_err(s1.cpu().numpy(), s1_o) < TOL_F32
+    # element by element as well, each against its own size with a floor far below the rms of the vector
+    assert float(np.max(np.abs(got - th_o) / np.maximum(np.abs(th_o), 1e-2))) < 1e-4
+
+
 def test_config3_full_size(sgdb, cuda_device):
     """P = 100 M, W = 208 (N = 200, b = 8), bf16 rows (41.6 GB), Adam, T = 5 steps."""
     _need_memory(cuda_device, 48)

@@ -4,7 +4,8 @@ Some users of the library run where cudaMalloc is not an option (all device memo
 another component's pool, or allocation is forbidden inside their serving loop).  For them the library
 carries a fixed staging array.  This test calls that entry point through the C ABI twice in a row and
 checks every output against sgdb_step_host, which uses a caller-supplied workspace; the two must agree
-within the tolerance of the other parity tests (they are in fact the same bits).  The file sorts last so
+within the tolerance of the other parity tests (they are in fact the same bits).  It also checks what the
+entry point is for: the amount of free device memory is the same before and after the second call.  The file sorts last so
 that a run that stops at the first failure has already run everything else; it also passes on its own.
 """
 import numpy as np
@@ -48,7 +49,13 @@ def test_static_scratch_step_matches_workspace_step_on_two_calls(sgdb, cuda_devi
         h_grad = wl.grad_matrix(seed, t, W, P, scales, dtype, "cpu", ld=ld)
         arrival, tags = step_inputs(seed, t, W, N)
         args = (h_grad, P, torch.from_numpy(arrival), torch.from_numpy(tags), t, N, W - N)
-        st_a = sgdb.sgdb_step_host_static(*args, theta_a, sa[0], sa[1], gpu_opt(OPTS[kind], t + 1), *out_a, ld=ld)
+        opt_a = gpu_opt(OPTS[kind], t + 1)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info(dev)[0]
+        st_a = sgdb.sgdb_step_host_static(*args, theta_a, sa[0], sa[1], opt_a, *out_a, ld=ld)
+        free_after = torch.cuda.mem_get_info(dev)[0]
+        if t > 0:  # the first call on a device may make the driver load the library's code; later calls take nothing
+            assert free_after == free_before, "the call without a workspace changed the free device memory"
         st_b = sgdb.sgdb_step_host(*args, theta_b, sb[0], sb[1], gpu_opt(OPTS[kind], t + 1), *out_b, ws, ld=ld)
         assert st_a == st_b == 0
         assert torch.equal(out_a[1], out_b[1]) and torch.equal(out_a[2], out_b[2])  # mask, order
