@@ -783,6 +783,8 @@ def main():
                     help="flat workloads: two-level aggregation (sgdb_step_grouped) with the workers spread over this many machines")
     ap.add_argument("--columns", type=int, default=0,
                     help="override P with a smaller column count (profiler captures); not the benchmark workload")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="override N, the number of gradients used per step (profiler captures); not the benchmark workload")
     ap.add_argument("--spread-steps", type=int, default=200, help="single steps timed one by one for the spread")
     ap.add_argument("--sustain-seconds", type=float, default=2.0, help="length of the sustained run")
     ap.add_argument("--cpu-steps", type=int, default=5, help="steps of the all-cores oracle leg")
@@ -794,6 +796,10 @@ def main():
         import dataclasses
 
         cfg = dataclasses.replace(cfg, P=args.columns, name=cfg.name + "_columns_%d" % args.columns)
+    if args.rows > 0:
+        import dataclasses
+
+        cfg = dataclasses.replace(cfg, N=args.rows, name=cfg.name + "_rows_%d" % args.rows)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
