@@ -48,7 +48,7 @@ NOMINAL_HBM_GBS = 8000.0
 
 # DRAM traffic of one fused-step launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
 # as bytes per algorithmic byte; valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"src_digest": "f559b579ce14cf57", "dram_bytes_per_algorithmic_byte": 0.9948}
+NCU_TRAFFIC = {"src_digest": "4208c3027d17c36b", "dram_bytes_per_algorithmic_byte": 0.9956}
 
 
 def kernel_source_digest() -> str:

@@ -12,7 +12,7 @@ The inputs stand in for the workloads of "Revisiting Distributed Synchronous SGD
   * a stale tag marks a gradient computed for the previous iteration, the only way
     Algorithm 4 meets a tag other than t;
   * W = N + b follows the paper's best split of 100 machines (N=96, b=4, Section 3.1)
-    and its 53/106/212-worker runs (Section 4.1).
+    and its 53/106/212-worker runs (Section 4.2, Appendix A.3).
 
 Small per-worker quantities come from numpy's Philox generator on the host; the
 large gradient matrices are drawn with torch's seeded generator on the device
