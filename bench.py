@@ -13,8 +13,9 @@ e2e       the same metric through sgdb_step_host: gradients, arrival times and t
 roofline  algorithmic bytes of a step (gradient rows + parameters and state read and written) over
           the measured step time, against the measured HBM copy bandwidth of this machine
 extra     (one GPU, default workload) the spread of single-step times, a sustained run of at least
-          two seconds with the clocks seen, the same step as three separate calls, and the other
-          four seeded workloads: tiny SGD, 300-tensor segmented, bf16 rows + Adam, arrival by arrival
+          two seconds with the clocks seen, the same step as three separate calls, its variants (with
+          the parameter average, with the time-out rule, two-level), and the other four seeded
+          workloads: tiny SGD, 300-tensor segmented, bf16 rows + Adam, arrival by arrival
 With --gpus N > 1 (under torchrun) every rank is one parameter-server shard holding its own P
 columns; there is no data-path collective, and the value is the sum over ranks over the slowest rank.
 --impl reference times the CPU oracle on the same workload (all host cores, column ranges split
@@ -427,11 +428,60 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
         return {"separate_calls_ms_per_step": ms, "separate_calls_total_gbs": moved / (ms * 1e-3) / 1e9,
                 "separate_calls_launches_per_step": 3}
 
+    def variants():
+        """The other forms of the fused step on the same matrix: with the parameter average, with the time-out
+        rule, and two-level (workers on machines of 4).  Each 20 steps after 3 warm-up steps."""
+        esize = grad.element_size()
+        state_bytes = 2 * (1 + n_state) * P * 4
+        out = {}
+        avg_v = theta.clone()
+
+        def ema_step(i):
+            opt.step = i + 1
+            sgdb.sgdb_step_ema(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, avg_v, 0.9999,
+                               mask, order, info)
+
+        ms = time_steps(ema_step, 20, 3)
+        out["parameter_average"] = rates(N * P * esize + state_bytes + 2 * P * 4, N * P * esize, ms)
+        del avg_v
+        dl = 1.6
+        order_w = torch.zeros(W, dtype=torch.int32, device=dev)
+        kept = float(np.mean([int(((wl.arrivals(cfg.seed, t, W) <= np.float32(dl)) & (wl.tags(cfg.seed, t, W, N) == t)).sum())
+                              for t in range(N_SETS)]))
+
+        def deadline_step(i):
+            opt.step = i + 1
+            sgdb.sgdb_step_deadline(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, dl, 1, theta, s0, s1, opt, mask,
+                                    order_w, info)
+
+        ms = time_steps(deadline_step, 20 - 20 % N_SETS + N_SETS, 3)  # whole rotations of the draws: the kept count varies
+        out["deadline_1.6s"] = dict(rates(int(kept * P * esize) + state_bytes, int(kept * P * esize), ms), mean_rows_kept=kept)
+        if W % 4 == 0:
+            m_all = W // 4
+            m_kept = N // 4
+            group = torch.from_numpy((np.arange(W) // 4).astype(np.int32)).to(dev)
+            group_order = torch.zeros(m_kept, dtype=torch.int32, device=dev)
+            info3 = torch.zeros(3, dtype=torch.int32, device=dev)
+            current = torch.zeros(W, dtype=torch.int32, device=dev)
+
+            def grouped_step(i):
+                opt.step = i + 1
+                sgdb.sgdb_step_grouped(grad, P, arr_d[i % N_SETS], current, group, 0, m_all, m_kept, theta, s0, s1, opt,
+                                       mask, group_order, order_w, info3)
+
+            ms = time_steps(grouped_step, 20, 3)
+            assert info3.cpu().tolist() == [m_all, 0, 4 * m_kept]
+            out["two_level"] = dict(rates(4 * m_kept * P * esize + state_bytes, 4 * m_kept * P * esize, ms),
+                                    machines=m_all, machines_kept=m_kept, rows_used=4 * m_kept)
+        assert info.cpu().tolist()[1] == 0 and bool(torch.isfinite(theta).all())
+        return out
+
     grad_bytes = int(kept_mean * P * grad.element_size())
     state = dict(grad=grad, theta=theta, s0=s0, s1=s1, opt=opt)
     total = grad_bytes + 2 * (1 + n_state) * P * 4 + (2 * P * 4 if ema else 0)
     return dict(step=step, check=check, grad_bytes=grad_bytes, total_bytes=total,
-                launches_per_step=1, kernel="stream_rows_kernel<%s, %s>%s (the step is this one launch)"
+                launches_per_step=1, variants=variants,
+                kernel="stream_rows_kernel<%s, %s>%s (the step is this one launch)"
                 % (cfg.grad_dtype, cfg.opt["kind"], " + parameter average" if ema else
                    (", two-level: %d machines, %d kept" % (machines, n_machines) if machines else "")), state=state,
                 extra={"parameter_average": True} if ema else {"machines": machines, "machines_kept": n_machines,
@@ -652,6 +702,7 @@ def run_native(args, cfg):
             sustained["step_us_times_sm_mhz"] = ms_sustained * 1e3 * sc["sm_mhz"]
         extra["sustained"] = sustained
         wk["check"]()
+        extra["variants"] = wk["variants"]()
 
     # ---- end to end: gradients start in pinned host memory, new parameters are read back
     flat = not cfg.segments and not cfg.name.startswith("c4")
@@ -701,7 +752,7 @@ def run_native(args, cfg):
     # ---- the other four seeded workloads, one after the other (each frees its memory before the next)
     if headline and not args.only_headline:
         del wk["state"], step
-        wk["step"] = wk["check"] = wk["extra"] = None
+        wk["step"] = wk["check"] = wk["extra"] = wk["variants"] = None
         release_device_memory()
         others = {}
         for index, name, steps in ((0, "c0", 200), (2, "c2", 20), (3, "c3", 10), (4, "c4", 5)):

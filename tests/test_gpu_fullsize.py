@@ -141,8 +141,8 @@ def test_config3_full_size(sgdb, cuda_device):
 
 def test_config2_full_size_segmented(sgdb, cuda_device):
     """300 tensors with log-uniform lengths in [64, 2^21], W = 54 (N = 50, b = 4), momentum SGD:
-    one launch over the device table vs the oracle (small tensors whole, large ones at sampled columns)
-    and vs one fused launch per tensor (bitwise)."""
+    one launch over the device table, which also keeps one parameter average per tensor, vs the oracle (small
+    tensors whole, large ones at sampled columns) and vs one fused launch per tensor (bitwise, parameters and state)."""
     _need_memory(cuda_device, 20)
     dev, cfg = cuda_device, wl.CONFIGS[2]
     W, N, kind = cfg.W, cfg.N, cfg.opt["kind"]
@@ -159,8 +159,12 @@ def test_config2_full_size_segmented(sgdb, cuda_device):
         samples.append(cols)
     twins = [(s[0].clone(), s[1].clone()) for s in segs]
     table = sgdb.make_segment_table(segs, dev)
+    avgs = [s[0].clone() for s in segs]  # one parameter average per tensor, kept by the same launch
+    ema_table = sgdb.make_pointer_table(avgs, dev)
+    alpha = 0.875
     th_o = [segs[i][0][to_dev(samples[i], dev)].cpu().numpy().astype(np.float64) for i in range(len(segs))]
     v_o = [np.zeros(len(c)) for c in samples]
+    avg_o = [x.copy() for x in th_o]
     mask, order, info = selection_buffers(W, N, dev)
     mask2, order2, info2 = selection_buffers(W, N, dev)
     for t in range(2):
@@ -169,8 +173,8 @@ def test_config2_full_size_segmented(sgdb, cuda_device):
                 wl.grad_matrix(cfg.seed + i, t, W, theta.numel(), scales, "f32", dev, ld=grad.stride(0), out=grad)
         arrival, tags = step_inputs(cfg.seed, t, W, N)
         a_d, t_d = to_dev(arrival, dev), to_dev(tags, dev)
-        sgdb.sgdb_step_segmented(table, len(segs), torch.float32, a_d, t_d, t, N, cfg.b, gpu_opt(cfg.opt, t + 1),
-                                 mask, order, info)
+        sgdb.sgdb_step_segmented_ema(table, ema_table, alpha, len(segs), torch.float32, a_d, t_d, t, N, cfg.b,
+                                     gpu_opt(cfg.opt, t + 1), mask, order, info)
         rc, mask_o, order_o, n_valid = oracle.select(arrival, tags, t, N, cfg.b)
         assert rc == oracle.OK and info.cpu().tolist() == [n_valid, 0]
         assert order.cpu().numpy().tolist() == order_o.tolist()
@@ -178,6 +182,7 @@ def test_config2_full_size_segmented(sgdb, cuda_device):
             cols_d = to_dev(samples[i], dev)
             sample = wl.as_oracle_array(grad.index_select(1, cols_d))
             mean = oracle.aggregate(sample, len(samples[i]), order_o)
+            oracle.ema(avg_o[i], th_o[i], alpha)  # the average takes in the parameters before the update
             oracle.update(th_o[i], v_o[i], None, mean, oracle_opt(cfg.opt, t + 1))
             if i % 10 == 0:  # one launch per tensor, every tenth tensor
                 sgdb.sgdb_step(grad, theta.numel(), a_d, t_d, t, N, cfg.b, twins[i][0], twins[i][1], None,
@@ -186,6 +191,8 @@ def test_config2_full_size_segmented(sgdb, cuda_device):
     got_v = np.concatenate([segs[i][1][to_dev(samples[i], dev)].cpu().numpy() for i in range(len(segs))])
     assert rel_err(got, np.concatenate(th_o)) < TOL_F32
     assert rel_err(got_v, np.concatenate(v_o)) < TOL_F32
+    got_avg = np.concatenate([avgs[i][to_dev(samples[i], dev)].cpu().numpy() for i in range(len(segs))])
+    assert rel_err(got_avg, np.concatenate(avg_o)) < TOL_F32
     for i in range(0, len(segs), 10):
         assert torch.equal(segs[i][0], twins[i][0]) and torch.equal(segs[i][1], twins[i][1]), i
 
@@ -230,4 +237,85 @@ def test_config4_full_size_accumulate_on_arrival(sgdb, cuda_device, b):
     mask, order, finfo = selection_buffers(W, N, dev)
     sgdb.sgdb_step(grad, P, to_dev(arrival, dev), to_dev(tags, dev), 0, N, b, theta_f, sf[0], sf[1], gpu_opt(cfg.opt),
                    mask, order, finfo)
+    assert torch.equal(theta, theta_f) and torch.equal(s0, sf[0]) and torch.equal(s1, sf[1])
+
+
+def test_config1_full_size_two_level(sgdb, cuda_device):
+    """The C1 matrix with its 100 workers on 25 machines of 4 and the first 24 messages used: the one-launch
+    two-level step against the oracle at sampled columns, three steps with a stale worker in each."""
+    _need_memory(cuda_device, 12)
+    dev, cfg = cuda_device, wl.CONFIGS[1]
+    W, P, kind, M, N = cfg.W, cfg.P, cfg.opt["kind"], 25, 24
+    group = (np.arange(W) // 4).astype(np.int32)
+    rng = np.random.default_rng(cfg.seed + 7)
+    cols = _sample_columns(P, rng)
+    cols_d = to_dev(cols, dev)
+    scales = wl.worker_scales(cfg.seed, W)
+    theta = wl.theta0(cfg.seed, P, dev)
+    s0, s1 = gpu_state(kind, P, dev)
+    th_o = theta[cols_d].cpu().numpy().astype(np.float64)
+    s0_o, s1_o = oracle_state(kind, len(cols))
+    mask = torch.full((W,), 255, dtype=torch.uint8, device=dev)
+    gorder = torch.full((N,), -7, dtype=torch.int32, device=dev)
+    order = torch.full((W,), -7, dtype=torch.int32, device=dev)
+    info = torch.full((3,), -7, dtype=torch.int32, device=dev)
+    grad = None
+    for t in range(3):
+        grad = wl.grad_matrix(cfg.seed, t, W, P, scales, cfg.grad_dtype, dev, out=grad)
+        arrival = wl.arrivals(cfg.seed, t, W)
+        tags = np.full(W, t, np.int32)
+        if t == 1:
+            tags[int(rng.integers(0, W))] = t - 1  # its machine's message does not count: exactly 24 are left
+        sgdb.sgdb_step_grouped(grad, P, to_dev(arrival, dev), to_dev(tags, dev), to_dev(group, dev), t, M, N, theta, s0, s1,
+                               gpu_opt(cfg.opt, t + 1), mask, gorder, order, info)
+        rc, mask_o, gorder_o, order_o, n_valid = oracle.step_grouped(
+            wl.as_oracle_array(grad.index_select(1, cols_d)), len(cols), arrival, tags, group, t, M, N, th_o, s0_o, s1_o,
+            oracle_opt(cfg.opt, t + 1))
+        assert rc == oracle.OK and info.cpu().tolist() == [n_valid, 0, 4 * N]
+        assert mask.cpu().numpy().tolist() == mask_o.tolist() and gorder.cpu().numpy().tolist() == gorder_o.tolist()
+        assert order.cpu().numpy()[: 4 * N].tolist() == order_o.tolist()
+    assert rel_err(theta[cols_d].cpu().numpy(), th_o) < TOL_F32
+    assert rel_err(s0[cols_d].cpu().numpy(), s0_o) < TOL_F32 and rel_err(s1[cols_d].cpu().numpy(), s1_o) < TOL_F32
+    assert bool(torch.isfinite(theta).all())
+
+
+def test_config4_full_size_arrivals_with_time_out(sgdb, cuda_device):
+    """P = 23.8 M, 100 workers, the time-out rule one gradient per call, then the close call: outcomes replayed by the
+    oracle, parameters at sampled columns against the oracle and on the whole vector against the fused time-out step."""
+    _need_memory(cuda_device, 14)
+    dev, cfg = cuda_device, wl.CONFIGS[4]
+    W, P, kind = cfg.W, cfg.P, cfg.opt["kind"]
+    seed = cfg.seed + 31
+    rng = np.random.default_rng(seed)
+    cols = _sample_columns(P, rng)
+    cols_d = to_dev(cols, dev)
+    grad = wl.grad_matrix(seed, 0, W, P, wl.worker_scales(seed, W), "f32", dev)
+    arrival, tags = step_inputs(seed, 0, W, 1)
+    deadline = float(np.float32(1.5))
+    theta = wl.theta0(seed, P, dev)
+    theta_f = theta.clone()
+    s0, s1 = gpu_state(kind, P, dev)
+    sf = gpu_state(kind, P, dev)
+    acc = torch.empty(P, device=dev)
+    counter = torch.zeros(4, dtype=torch.int32, device=dev)
+    info = torch.zeros(2, dtype=torch.int32, device=dev)
+    th_o = theta[cols_d].cpu().numpy().astype(np.float64)
+    s0_o, s1_o = oracle_state(kind, len(cols))
+    acc_o, state_o = np.zeros(len(cols)), oracle.new_server_state()
+    sample = wl.as_oracle_array(grad.index_select(1, cols_d))
+    kept = 0
+    for w in wl.delivery_sequence(arrival):
+        sgdb.sgdb_accumulate_arrival_deadline(grad[w], int(tags[w]), float(arrival[w]), 0, deadline, acc, counter, info)
+        want = oracle.accumulate_arrival_deadline(sample[w], int(tags[w]), float(arrival[w]), 0, deadline, acc_o, state_o)
+        assert info.cpu().tolist()[0] == want
+        kept += want
+    assert 20 < kept < W and counter.cpu().tolist() == [kept, W, 0, 0]
+    sgdb.sgdb_accumulate_close(0, 1, acc, counter, theta, s0, s1, gpu_opt(cfg.opt), info)
+    rc, outcome = oracle.accumulate_close(0, 1, acc_o, state_o, th_o, s0_o, s1_o, oracle_opt(cfg.opt))
+    assert rc == oracle.OK and outcome == 2 and info.cpu().tolist() == [2, kept] and counter.cpu().tolist() == [0, W, 0, 1]
+    assert rel_err(theta[cols_d].cpu().numpy(), th_o) < TOL_F32 and rel_err(s0[cols_d].cpu().numpy(), s0_o) < TOL_F32
+    mask, order, finfo = selection_buffers(W, W, dev)
+    sgdb.sgdb_step_deadline(grad, P, to_dev(arrival, dev), to_dev(tags, dev), 0, deadline, 1, theta_f, sf[0], sf[1],
+                            gpu_opt(cfg.opt), mask, order, finfo)
+    assert finfo.cpu().tolist() == [kept, 0]
     assert torch.equal(theta, theta_f) and torch.equal(s0, sf[0]) and torch.equal(s1, sf[1])
