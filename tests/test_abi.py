@@ -96,6 +96,28 @@ def test_host_checkable_errors_return_before_any_launch(lib):
     assert need >= 6 * 12 * 4
     assert lib.sgdb_set_tuning(i32(1000), i32(0)) == INVALID
     assert lib.sgdb_set_tuning(i32(0), i32(0)) == 0
+    assert lib.sgdb_set_arrival_tuning(i64(0), i32(9)) == INVALID
+    assert lib.sgdb_set_arrival_tuning(i64(-1), i32(0)) == 0
+    f32 = ctypes.c_float
+    # two-level selection: W, M, N out of range
+    for W, M, N in ((0, 1, 1), (4, 0, 1), (4, 2, 0), (4, 2, 3), (1025, 2, 1), (4, 1025, 1)):
+        assert lib.sgdb_select_grouped(one, one, one, i32(0), i32(W), i32(M), i32(N), one, one, one, one, null) == INVALID
+    assert lib.sgdb_select_grouped(one, one, null, i32(0), i32(4), i32(2), i32(1), one, one, one, one, null) == INVALID
+    # time-out rule: NaN deadline, n_min out of range
+    assert lib.sgdb_select_deadline(one, one, i32(0), i32(4), f32(float("nan")), i32(1), one, one, one, null) == INVALID
+    assert lib.sgdb_step_segmented_deadline(one, i32(1), i32(0), one, one, i32(0), i32(4), f32(1.0), i32(5), null, one, one,
+                                            one, null) == INVALID
+    # an arriving row at an address that is not a multiple of its element size; a close call without n_min
+    assert lib.sgdb_accumulate_arrival_deadline(ctypes.c_void_p(18), i32(0), i32(0), f32(1.0), i32(0), f32(2.0), i64(8), one,
+                                                one, one, null) == INVALID
+    assert lib.sgdb_accumulate_arrival_deadline(one, i32(0), i32(0), f32(1.0), i32(0), f32(float("nan")), i64(8), one, one,
+                                                one, null) == INVALID
+    assert lib.sgdb_accumulate_close(i32(0), i32(0), i64(8), one, one, one, null, null, null, null, f32(0.0), one, null) == INVALID
+    # per-tensor averages: the pointer table and alpha
+    assert lib.sgdb_step_segmented_ema(one, null, f32(0.5), i32(1), i32(0), one, one, i32(0), i32(1), i32(0), null, one, one,
+                                       one, null) == INVALID
+    assert lib.sgdb_step_segmented_ema(one, one, f32(1.5), i32(1), i32(0), one, one, i32(0), i32(1), i32(0), null, one, one,
+                                       one, null) == INVALID
 
 
 def test_learning_rate_schedule_is_a_host_computation(lib):

@@ -225,3 +225,28 @@ def test_grouped_step_mid_size_many_machines(sgdb, cuda_device):
     assert gorder.cpu().numpy().tolist() == gorder_o.tolist() and order.cpu().numpy()[:96].tolist() == order_o.tolist()
     assert rel_err(theta[cols_d].cpu().numpy(), th_o) < TOL_F32 and rel_err(s0[cols_d].cpu().numpy(), s0_o) < TOL_F32
     assert bool(torch.isfinite(theta).all())
+
+
+@pytest.mark.parametrize("W,M,N", [(1024, 256, 200), (1000, 1000, 999), (37, 37, 37)])
+def test_grouped_step_at_the_largest_counts(sgdb, cuda_device, W, M, N):
+    """As many workers and machines as the library accepts (and every machine kept): selection words bit-exact,
+    parameters within tolerance."""
+    dev = cuda_device
+    P, seed = 6000, 191
+    rng = np.random.default_rng(seed + W)
+    group = rng.permutation(np.arange(W) % M).astype(np.int32)
+    grad = wl.grad_matrix(seed, 0, W, P, wl.worker_scales(seed, W), "f32", dev)
+    arrival = wl.arrivals(seed, 0, W)
+    arrival[: W // 8] = arrival[W // 8: 2 * (W // 8)]  # plenty of equal times
+    tags = np.zeros(W, np.int32)
+    theta = wl.theta0(seed, P, dev)
+    th_o = theta.cpu().numpy().astype(np.float64)
+    mask, gorder, order, info = _buffers(W, N, dev)
+    sgdb.sgdb_step_grouped(grad, P, to_dev(arrival, dev), to_dev(tags, dev), to_dev(group, dev), 0, M, N, theta, None, None,
+                           gpu_opt(OPTS["sgd"]), mask, gorder, order, info)
+    rc, mask_o, gorder_o, order_o, n_valid = oracle.step_grouped(wl.as_oracle_array(grad), P, arrival, tags, group, 0, M, N,
+                                                                 th_o, None, None, oracle_opt(OPTS["sgd"]))
+    assert rc == oracle.OK and info.cpu().tolist() == [n_valid, 0, len(order_o)]
+    assert mask.cpu().numpy().tolist() == mask_o.tolist() and gorder.cpu().numpy().tolist() == gorder_o.tolist()
+    assert order.cpu().numpy()[: len(order_o)].tolist() == order_o.tolist()
+    assert rel_err(theta.cpu().numpy(), th_o) < TOL_F32
