@@ -35,7 +35,9 @@
  *   - Base pointers of G, theta, state, mean and acc must be 16-byte aligned in
  *     the flat calls.  Rows are streamed with 16-byte bulk copies when
  *     ld * sizeof(element) is a multiple of 16; any other ld is accepted and
- *     takes an element-wise load path with identical results.
+ *     takes an element-wise load path with identical results.  On the 16-byte path
+ *     the padding columns of a kept row up to the next 16-byte boundary after its last
+ *     used column may be read; their values are never used.
  *   - Summation order is fixed: the kept rows are added one after another in
  *     arrival order, starting from +0, in fp32, and the sum is divided by N once.
  *     Results are therefore bit-reproducible run to run and identical between

@@ -284,9 +284,12 @@ __global__ void __launch_bounds__(1024) select_grouped_kernel(const float* __res
 // the next tile's rows are already in flight while this tile's epilogue runs.
 //
 // Bulk copies need 16-byte aligned addresses and sizes.  A segment whose gradient
-// base or row pitch is not 16-byte aligned, and the last (< 16 byte) sliver of a
-// ragged tile, are read with ordinary element loads by the consumers instead; the
-// additions happen in the same order either way.
+// base or row pitch is not 16-byte aligned is read with ordinary element loads by
+// the consumers instead; the additions happen in the same order either way.  With
+// an aligned pitch the last 16-byte chunk of a ragged tile is copied whole: the
+// columns between len and the next multiple of 16 bytes are padding inside the row
+// pitch (or at least inside the same 16-byte block as the last valid element), they
+// are read and never used.
 
 struct StreamParams {
   const sgdb_segment_t* table;  // device segment table, or nullptr: use `flat`
@@ -335,7 +338,7 @@ struct TileDesc {
   float* s1;
   long long ld;
   int ncols;      // valid columns in the tile
-  int bulk_cols;  // leading columns delivered by bulk copy (0: none)
+  int bulk_cols;  // leading columns delivered by bulk copy (0: none); may exceed ncols by the row's padding
   bool vec_ok;    // theta/state slices may be accessed 16 bytes at a time
   bool bad;       // a pointer this rule needs is null in the segment table: the tile is skipped
 };
@@ -385,7 +388,9 @@ __device__ __forceinline__ TileDesc<GT> locate_tile(const StreamParams& p, const
   td.ncols = rest < TILE ? static_cast<int>(rest) : TILE;
   const bool bulk_ok = ((reinterpret_cast<uintptr_t>(seg.grad) & 15u) == 0) &&
                        (((seg.ld * static_cast<long long>(sizeof(GT))) & 15) == 0);
-  td.bulk_cols = bulk_ok ? (td.ncols / V) * V : 0;
+  // A 16-byte aligned row pitch leaves room for the whole last 16-byte chunk of a ragged tile (ld is a multiple
+  // of V and ld >= len): the copy takes it along, padding included; lanes beyond ncols are never stored.
+  td.bulk_cols = bulk_ok ? ((td.ncols + V - 1) / V) * V : 0;
   td.bad = false;
   td.ema = ema != nullptr ? ema + col0 : nullptr;
   td.vec_ok = (((reinterpret_cast<uintptr_t>(seg.theta) | reinterpret_cast<uintptr_t>(seg.state0) |
