@@ -304,6 +304,66 @@ sgdb_status_t sgdb_step_grouped(const void *d_grad, sgdb_dtype_t dt, int64_t P, 
                                 int32_t *d_group_order, int32_t *d_order, int32_t *d_info, void *stream);
 
 /*
+ * sgdb_step_rows, sgdb_step_rows_ordered, sgdb_shard_range -- the step as ONE of several
+ * parameter servers runs it (Section 1.1: the parameters are split over servers, server j holds
+ * theta[j], receives every worker's gradient of theta[j] and hands theta[j] back to the workers;
+ * Algorithm 4 runs on every server; Algorithm 3 sends G[j] to server j and reads theta[j] from it).
+ * This is the form for several GPUs: each GPU is server j for one range of columns, the workers'
+ * gradients are whole rows that live in any GPU's memory, and every GPU keeps a full copy of theta
+ * for its workers to read.
+ *
+ *   d_rows     [W] DEVICE array of device addresses: d_rows[w] = column `first` of worker w's
+ *                  gradient, i.e. the first element server j is responsible for; `len` elements of
+ *                  type dt are read from the kept rows, the others are never touched.  An address
+ *                  may belong to this GPU or to a peer GPU whose memory is mapped into this process.
+ *                  Element-aligned addresses are required; when every kept row is 16-byte aligned
+ *                  the rows are pulled with bulk copies (never multicast), else with element loads,
+ *                  same results.
+ *   len            columns of this server's range (sgdb_shard_range gives ranges that keep every
+ *                  server's addresses 16-byte aligned when the full rows are)
+ *   d_theta, d_state0, d_state1 [len]  this server's range of the parameters and state, in/out,
+ *                  this GPU's memory, 16-byte aligned
+ *   d_replicas [R] DEVICE array of device addresses, R <= SGDB_MAX_REPLICAS, or NULL with R = 0:
+ *                  d_replicas[r] = where copy r of this range lives (column `first` of a full copy
+ *                  of theta, this GPU's memory or a peer's); the new parameters are stored to
+ *                  d_theta and to every replica in the same pass (4 * R more bytes per column)
+ *   selection      sgdb_step_rows takes it in the kernel's prologue like sgdb_step (d_arrival,
+ *                  d_tags, t, N, b in; d_mask, d_order, d_info out): every server computes the same
+ *                  selection from the same W numbers, so all ranges use the same N gradients.
+ *                  sgdb_step_rows_ordered is given it: d_order [N] row ids in summation sequence
+ *                  (each in [0, W)), d_info [2] in/out -- when d_info[1] != SGDB_OK on entry nothing
+ *                  is done; the mean divides by N.
+ * A null or misaligned address among the kept rows or the replicas, or a row id outside [0, W),
+ * makes the kernel touch nothing and write SGDB_ERR_INVALID_ARG to d_info[1].
+ * Summation order, arithmetic and therefore the bits of theta and state are those of sgdb_step on
+ * the same columns.  One launch; no block waits for another GPU.  Ordering between GPUs is the
+ * caller's: every kept gradient must be complete before the launch, and a replica may be read only
+ * after the launches of all servers that write to it have completed (the barrier of the
+ * synchronous protocol, Section 3).
+ *
+ * sgdb_step_rows_ordered also serves two-level aggregation across GPUs (Section 6, see
+ * sgdb_step_grouped): each machine writes the mean of its workers' gradients (sgdb_select over its own
+ * workers, then sgdb_aggregate), the servers then take the kept machines' means as rows, with
+ * d_order = the d_group_order of sgdb_select_grouped; the result has the bits of sgdb_step_grouped.
+ *
+ * sgdb_shard_range (host computation): range j of n_servers over P columns, contiguous, in order,
+ * together covering [0, P), every start a multiple of SGDB_SHARD_ALIGN columns; trailing ranges
+ * may be empty.
+ */
+#define SGDB_MAX_REPLICAS 64 /* largest accepted R */
+#define SGDB_SHARD_ALIGN 64  /* columns; keeps fp32 and bf16 rows 128-byte aligned at every range start */
+sgdb_status_t sgdb_step_rows(const void *const *d_rows, sgdb_dtype_t dt, int64_t len,
+                             const float *d_arrival, const int32_t *d_tags, int32_t t, int32_t N,
+                             int32_t b, float *d_theta, float *d_state0, float *d_state1,
+                             const sgdb_opt_t *opt, float *const *d_replicas, int32_t R,
+                             uint8_t *d_mask, int32_t *d_order, int32_t *d_info, void *stream);
+sgdb_status_t sgdb_step_rows_ordered(const void *const *d_rows, int32_t W, sgdb_dtype_t dt, int64_t len,
+                                     int32_t N, const int32_t *d_order, int32_t *d_info, float *d_theta,
+                                     float *d_state0, float *d_state1, const sgdb_opt_t *opt,
+                                     float *const *d_replicas, int32_t R, void *stream);
+sgdb_status_t sgdb_shard_range(int64_t P, int32_t n_servers, int32_t j, int64_t *first, int64_t *len);
+
+/*
  * sgdb_accumulate_arrival -- Algorithm 4's inner loop taken literally: one
  * gradient per call, in the order the gradients reach the server.
  *

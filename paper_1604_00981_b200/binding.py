@@ -28,8 +28,11 @@ EXPORTS = (
     "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_accumulate_arrival_ema", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
     "sgdb_select_grouped", "sgdb_step_grouped", "sgdb_step_segmented_ema", "sgdb_step_segmented_deadline",
     "sgdb_accumulate_arrival_deadline", "sgdb_accumulate_close", "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version",
+    "sgdb_step_rows", "sgdb_step_rows_ordered", "sgdb_shard_range",
 )
 SGDB_STATIC_SCRATCH_BYTES = 8 << 20
+SGDB_MAX_REPLICAS = 64
+SGDB_SHARD_ALIGN = 64
 
 
 class SgdbError(RuntimeError):
@@ -104,6 +107,10 @@ def _load():
         "sgdb_select_grouped": (i32, [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]),
         "sgdb_step_grouped": (i32, [vp, i32, i64, i64, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt),
                                     vp, vp, vp, vp, vp]),
+        "sgdb_step_rows": (i32, [vp, i32, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt), vp, i32,
+                                 vp, vp, vp, vp]),
+        "sgdb_step_rows_ordered": (i32, [vp, i32, i32, i64, i32, vp, vp, vp, vp, vp, ctypes.POINTER(_COpt), vp, i32, vp]),
+        "sgdb_shard_range": (i32, [i64, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]),
         "sgdb_accumulate_arrival": (i32, [vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, ctypes.POINTER(_COpt), vp, vp]),
         "sgdb_accumulate_arrival_ema": (i32, [vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, ctypes.POINTER(_COpt), vp,
                                               ctypes.c_float, vp, vp]),
@@ -368,6 +375,49 @@ def sgdb_step_grouped(grad, P: int, arrival, tags, group, t: int, M: int, N: int
                                   ctypes.byref(c), _dev(mask, torch.uint8, "mask"),
                                   _dev(group_order, torch.int32, "group_order"), _dev(order, torch.int32, "order"),
                                   _dev(info, torch.int32, "info"), _stream(stream)), "sgdb_step_grouped")
+
+
+def make_address_table(addresses, device) -> torch.Tensor:
+    """Device array of device addresses (int64 CUDA tensor) from integers, e.g. tensor.data_ptr() plus a byte
+    offset, or the address of a peer GPU's buffer mapped into this process.  The caller keeps the memory alive."""
+    return torch.tensor([int(a) for a in addresses], dtype=torch.int64).to(device)
+
+
+def sgdb_step_rows(rows, grad_dtype, length: int, arrival, tags, t: int, N: int, b: int, theta, state0, state1, opt: Opt,
+                   replicas, mask, order, info, stream=None) -> None:
+    """The fused step of one parameter server over its range of `length` columns: rows i64[W] holds the address of
+    each worker's gradient at the range's first column (make_address_table), replicas i64[R] or None the addresses
+    the new parameters are also stored to."""
+    dt = SGDB_BF16 if grad_dtype == torch.bfloat16 else SGDB_F32
+    R = 0 if replicas is None else replicas.numel()
+    c = opt._c()
+    _check(_lib.sgdb_step_rows(_dev(rows, torch.int64, "rows"), dt, length, _dev(arrival, torch.float32, "arrival"),
+                               _dev(tags, torch.int32, "tags"), t, N, b, _dev(theta, torch.float32, "theta"),
+                               _dev(state0, torch.float32, "state0"), _dev(state1, torch.float32, "state1"),
+                               ctypes.byref(c), _dev(replicas, torch.int64, "replicas"), R,
+                               _dev(mask, torch.uint8, "mask"), _dev(order, torch.int32, "order"),
+                               _dev(info, torch.int32, "info"), _stream(stream)), "sgdb_step_rows")
+
+
+def sgdb_step_rows_ordered(rows, grad_dtype, length: int, N: int, order, info, theta, state0, state1, opt: Opt,
+                           replicas, stream=None) -> None:
+    """sgdb_step_rows with the selection given: order i32[N] row ids in summation sequence, info i32[2] in/out."""
+    dt = SGDB_BF16 if grad_dtype == torch.bfloat16 else SGDB_F32
+    R = 0 if replicas is None else replicas.numel()
+    c = opt._c()
+    _check(_lib.sgdb_step_rows_ordered(_dev(rows, torch.int64, "rows"), rows.numel(), dt, length, N,
+                                       _dev(order, torch.int32, "order"), _dev(info, torch.int32, "info"),
+                                       _dev(theta, torch.float32, "theta"), _dev(state0, torch.float32, "state0"),
+                                       _dev(state1, torch.float32, "state1"), ctypes.byref(c),
+                                       _dev(replicas, torch.int64, "replicas"), R, _stream(stream)),
+           "sgdb_step_rows_ordered")
+
+
+def sgdb_shard_range(P: int, n_servers: int, j: int):
+    """(first column, number of columns) of parameter server j out of n_servers over P columns (host computation)."""
+    first, length = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(_lib.sgdb_shard_range(P, n_servers, j, ctypes.byref(first), ctypes.byref(length)), "sgdb_shard_range")
+    return int(first.value), int(length.value)
 
 
 def sgdb_accumulate_arrival(row, row_tag: int, t: int, N: int, acc, counter, theta, state0, state1,

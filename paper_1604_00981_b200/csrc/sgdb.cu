@@ -154,7 +154,7 @@ sgdb_status_t check_selection_args(const void* arrival, const void* tags, int32_
 
 // ---------------------------------------------------------------- row-streaming launch
 
-template <typename GT, int EP, bool GROUPED = false>
+template <typename GT, int EP, bool GROUPED = false, bool ROWS = false>
 sgdb_status_t launch_stream_t(const StreamParams& p_in, cudaStream_t stream) {
   const DeviceInfo* dev = nullptr;
   sgdb_status_t st = device_info(&dev);
@@ -162,13 +162,14 @@ sgdb_status_t launch_stream_t(const StreamParams& p_in, cudaStream_t stream) {
   StreamParams p = p_in;
   constexpr int kCH = Shape<GT>::kCH;
   constexpr int kStageBytes = kNT * kCH * 16;
-  auto kernel = stream_rows_kernel<GT, EP, kNT, kCH, GROUPED>;
+  auto kernel = stream_rows_kernel<GT, EP, kNT, kCH, GROUPED, ROWS>;
 
   // shared memory: ring + 2 barriers per slot + order[N] + tile prefix[S + 1] + selection scratch
   if (p.order_cap < p.N) p.order_cap = p.N;
   const size_t fixed = static_cast<size_t>((p.order_cap + 3) & ~3) * 4 + (p.table ? (static_cast<size_t>(p.S) + 1) * 4 : 0) +
                        (p.arrival ? static_cast<size_t>(p.W) * 4 : 0) +
-                       (GROUPED ? (4 * static_cast<size_t>(p.M) + static_cast<size_t>(p.N) + 1) * 4 : 0) + 16;
+                       (GROUPED ? (4 * static_cast<size_t>(p.M) + static_cast<size_t>(p.N) + 1) * 4 : 0) +
+                       (ROWS ? (static_cast<size_t>(p.order_cap) + static_cast<size_t>(p.R)) * 8 : 0) + 16;
   int ctas_per_sm = g_ctas_per_sm;
   int stages = g_stages;
   const size_t per_sm_budget = static_cast<size_t>(dev->max_smem_optin);
@@ -230,6 +231,22 @@ sgdb_status_t launch_stream_grouped_ep(int ep, const StreamParams& p, cudaStream
 
 sgdb_status_t launch_stream_grouped(int dt, int ep, const StreamParams& p, cudaStream_t stream) {
   return dt == SGDB_BF16 ? launch_stream_grouped_ep<BF16>(ep, p, stream) : launch_stream_grouped_ep<float>(ep, p, stream);
+}
+
+template <typename GT>
+sgdb_status_t launch_stream_rows_ep(int ep, const StreamParams& p, cudaStream_t stream) {
+  switch (ep) {
+    case EP_SGD: return launch_stream_t<GT, EP_SGD, false, true>(p, stream);
+    case EP_MOMENTUM: return launch_stream_t<GT, EP_MOMENTUM, false, true>(p, stream);
+    case EP_RMSPROP: return launch_stream_t<GT, EP_RMSPROP, false, true>(p, stream);
+    case EP_ADAM: return launch_stream_t<GT, EP_ADAM, false, true>(p, stream);
+    case EP_ADAGRAD: return launch_stream_t<GT, EP_ADAGRAD, false, true>(p, stream);
+  }
+  return SGDB_ERR_INVALID_ARG;
+}
+
+sgdb_status_t launch_stream_rows(int dt, int ep, const StreamParams& p, cudaStream_t stream) {
+  return dt == SGDB_BF16 ? launch_stream_rows_ep<BF16>(ep, p, stream) : launch_stream_rows_ep<float>(ep, p, stream);
 }
 
 long long tiles_of(int dt, long long len) {
@@ -576,6 +593,30 @@ sgdb_status_t sgdb_step_grouped(const void* d_grad, sgdb_dtype_t dt, int64_t P, 
   return launch_stream_grouped(dt, ep, p, static_cast<cudaStream_t>(stream));
 }
 
+// Checks and kernel parameters shared by the two forms of the step whose rows are given by address;
+// the selection fields are filled in by the caller.  `ep` receives the epilogue selector.
+static sgdb_status_t prepare_rows(const void* const* d_rows, int32_t W, sgdb_dtype_t dt, int64_t len, int32_t N,
+                                  float* d_theta, float* d_state0, float* d_state1, const sgdb_opt_t* opt,
+                                  float* const* d_replicas, int32_t R, StreamParams* p, int* ep) {
+  if (d_rows == nullptr || !dtype_ok(dt) || len < 0 || N < 1 || W < N || W > SGDB_MAX_WORKERS) return SGDB_ERR_INVALID_ARG;
+  if (R < 0 || R > SGDB_MAX_REPLICAS || (R > 0 && d_replicas == nullptr)) return SGDB_ERR_INVALID_ARG;
+  if (tiles_of(dt, len) > 0x7fffffffLL) return SGDB_ERR_UNSUPPORTED;
+  Hyper h;
+  sgdb_status_t st = prepare_rule(opt, d_state0, d_state1, &h, ep);
+  if (st != SGDB_OK) return st;
+  if (d_theta == nullptr || !is_aligned16(d_theta) || !is_aligned16(d_state0) || !is_aligned16(d_state1))
+    return SGDB_ERR_INVALID_ARG;
+  *p = flat_params(d_theta, d_state0, d_state1, nullptr, 0, len, N);
+  p->rows = d_rows;
+  p->W_rows = W;
+  p->replicas = d_replicas;
+  p->R = R;
+  p->h = h;
+  p->order_cap = N;
+  p->deadline = kNoDeadline;
+  return SGDB_OK;
+}
+
 static sgdb_status_t arrival(const void* d_row, sgdb_dtype_t dt, int32_t row_tag, int32_t t, int32_t N, int64_t P,
                              float* d_acc, int32_t* d_counter, float* d_theta, float* d_state0, float* d_state1,
                              const sgdb_opt_t* opt, float* d_ema, float alpha, int32_t* d_info, void* stream) {
@@ -693,6 +734,52 @@ sgdb_status_t sgdb_accumulate_close(int32_t t, int32_t n_min, int64_t P, const f
     case EP_ADAGRAD: return launch_on_server_state(close_iteration_kernel<EP_ADAGRAD>, g, p, s);
   }
   return SGDB_ERR_INVALID_ARG;
+}
+
+sgdb_status_t sgdb_step_rows(const void* const* d_rows, sgdb_dtype_t dt, int64_t len, const float* d_arrival,
+                             const int32_t* d_tags, int32_t t, int32_t N, int32_t b, float* d_theta, float* d_state0,
+                             float* d_state1, const sgdb_opt_t* opt, float* const* d_replicas, int32_t R,
+                             uint8_t* d_mask, int32_t* d_order, int32_t* d_info, void* stream) {
+  sgdb_status_t st = check_selection_args(d_arrival, d_tags, N, b, d_mask, d_order, d_info);
+  if (st != SGDB_OK) return st;
+  StreamParams p{};
+  int ep = 0;
+  st = prepare_rows(d_rows, N + b, dt, len, N, d_theta, d_state0, d_state1, opt, d_replicas, R, &p, &ep);
+  if (st != SGDB_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (len == 0) return launch_select(d_arrival, d_tags, t, N, b, d_mask, d_order, d_info, s);
+  set_in_kernel_selection(&p, d_arrival, d_tags, t, N + b, d_mask, d_order, d_info);
+  return launch_stream_rows(dt, ep, p, s);
+}
+
+sgdb_status_t sgdb_step_rows_ordered(const void* const* d_rows, int32_t W, sgdb_dtype_t dt, int64_t len, int32_t N,
+                                     const int32_t* d_order, int32_t* d_info, float* d_theta, float* d_state0,
+                                     float* d_state1, const sgdb_opt_t* opt, float* const* d_replicas, int32_t R,
+                                     void* stream) {
+  if (d_order == nullptr || d_info == nullptr) return SGDB_ERR_INVALID_ARG;
+  StreamParams p{};
+  int ep = 0;
+  sgdb_status_t st = prepare_rows(d_rows, W, dt, len, N, d_theta, d_state0, d_state1, opt, d_replicas, R, &p, &ep);
+  if (st != SGDB_OK) return st;
+  if (len == 0) return SGDB_OK;
+  p.order = d_order;
+  p.info = d_info;
+  p.status_out = d_info + 1;
+  return launch_stream_rows(dt, ep, p, static_cast<cudaStream_t>(stream));
+}
+
+sgdb_status_t sgdb_shard_range(int64_t P, int32_t n_servers, int32_t j, int64_t* first, int64_t* len) {
+  if (first == nullptr || len == nullptr || P < 0 || P > (INT64_MAX >> 1) || n_servers < 1 || j < 0 || j >= n_servers)
+    return SGDB_ERR_INVALID_ARG;
+  const int64_t a = SGDB_SHARD_ALIGN;
+  const int64_t per = (P + n_servers - 1) / n_servers;
+  const int64_t chunk = (per + a - 1) / a * a;
+  const int64_t start = static_cast<int64_t>(j) * chunk;  // at most P + n_servers * (a + 1): no overflow
+  const int64_t lo = start < P ? start : P;
+  const int64_t rest = P - lo;
+  *first = lo;
+  *len = rest < chunk ? rest : chunk;
+  return SGDB_OK;
 }
 
 // Workspace layout of sgdb_step_host: arrival[W] f32 | tags[W] i32 | order[N] i32 | info[2] i32 |

@@ -326,6 +326,14 @@ struct StreamParams {
   float* ema;
   float* const* ema_table;
   float ema_alpha, ema_one_minus_alpha;
+  // Rows by address (ROWS kernels): the gradient of worker w starts at rows[w] (W_rows entries, this GPU's
+  // memory or a peer's, mapped into this process) instead of at flat.grad + w * ld; column i of this server's
+  // shard is element i of every row, of flat.theta and of the state.  The new parameters are also stored to
+  // replicas[0 .. R): the copies of this shard that the workers read (this GPU's or a peer's memory).
+  const void* const* rows;
+  int32_t W_rows;
+  float* const* replicas;
+  int32_t R;
   Hyper h;
 };
 
@@ -405,7 +413,13 @@ __device__ __forceinline__ TileDesc<GT> locate_tile(const StreamParams& p, const
 
 // GROUPED: the kept rows fall into runs (one per kept machine); every run is summed on its own,
 // divided by its length, and the runs' means are added in sequence and divided by their number.
-template <typename GT, int EP, int NT, int CH, bool GROUPED = false>
+// ROWS: every row has an address of its own (a table of pointers, peers' memory allowed) and the new
+// parameters are also stored to a list of replicas; this is the form a parameter server takes when the
+// workers' gradients live in other GPUs' memory: it pulls its columns of the kept rows with the same
+// bulk copies (never multicast) and pushes its shard of theta back with ordinary stores.  No block
+// waits for another GPU: the caller orders the launches of different GPUs (gradients complete before,
+// replicas complete after).
+template <typename GT, int EP, int NT, int CH, bool GROUPED = false, bool ROWS = false>
 __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamParams p) {
   using Tr = GradTraits<GT>;
   using Rule = RuleTraits<EP>;
@@ -424,7 +438,11 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
   int N = p.N;  // rows to add; with the time-out rule the selection below decides it
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + static_cast<size_t>(stages) * STAGE_BYTES);
   uint64_t* empty_bar = full_bar + stages;
-  int* order_s = reinterpret_cast<int*>(empty_bar + stages);
+  // ROWS: the kept rows' addresses in summation order, then the replicas' addresses
+  uint64_t* after_bars = empty_bar + stages;
+  const GT** rowptr_s = reinterpret_cast<const GT**>(after_bars);
+  float** repl_s = reinterpret_cast<float**>(after_bars + (ROWS ? p.order_cap : 0));
+  int* order_s = reinterpret_cast<int*>(after_bars + (ROWS ? p.order_cap + p.R : 0));
   int* prefix_s = order_s + ((p.order_cap + 3) & ~3);
   float* key_s = reinterpret_cast<float*>(prefix_s + (p.table != nullptr ? p.S + 1 : 0));
   int* gend_s = nullptr;  // GROUPED: rows of the machine of rank r are order_s[gend_s[r] .. gend_s[r + 1])
@@ -451,6 +469,37 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
   } else {
     if (p.info != nullptr && p.info[1] != SGDB_OK) return;
     for (int i = tid; i < N; i += NT + 32) order_s[i] = p.order[i];
+  }
+  bool rows_bulk = false;   // ROWS: every kept row starts on a 16-byte boundary
+  bool repl_vec = true;     // ROWS: every replica starts on a 16-byte boundary
+  if constexpr (ROWS) {
+    __syncthreads();  // order_s is complete
+    // bit 0: an address or a row id the kernel must not use; bit 1: a row off the 16-byte grid;
+    // bit 2: a replica off the 16-byte grid
+    int flags = 0;
+    for (int k = tid; k < N; k += NT + 32) {
+      const int w = order_s[k];
+      const GT* row = nullptr;
+      if (w >= 0 && w < p.W_rows) row = static_cast<const GT*>(p.rows[w]);
+      rowptr_s[k] = row;
+      const uintptr_t a = reinterpret_cast<uintptr_t>(row);
+      if (row == nullptr || (a & (sizeof(GT) - 1)) != 0) flags |= 1;
+      if ((a & 15u) != 0) flags |= 2;
+    }
+    for (int r = tid; r < p.R; r += NT + 32) {
+      float* dst = p.replicas[r];
+      repl_s[r] = dst;
+      const uintptr_t a = reinterpret_cast<uintptr_t>(dst);
+      if (dst == nullptr || (a & 3u) != 0) flags |= 1;
+      if ((a & 15u) != 0) flags |= 4;
+    }
+    const bool unusable = __syncthreads_or(flags & 1) != 0;  // (the call returns a truth value, not the bits)
+    rows_bulk = __syncthreads_or(flags & 2) == 0;
+    repl_vec = __syncthreads_or(flags & 4) == 0;
+    if (unusable) {  // nothing is touched; every block takes the same decision
+      if (blockIdx.x == 0 && tid == 0 && p.status_out != nullptr) *p.status_out = SGDB_ERR_INVALID_ARG;
+      return;
+    }
   }
   if (tid == 0) {
     s_abort = 0;
@@ -503,7 +552,8 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
       int s = 0;
       uint32_t phase = 0;
       for (int tile = blockIdx.x; tile < total_tiles && !timed_out; tile += gridDim.x) {
-        const TileDesc<GT> td = locate_tile<GT, TILE, EP>(p, prefix_s, tile);
+        TileDesc<GT> td = locate_tile<GT, TILE, EP>(p, prefix_s, tile);
+        if constexpr (ROWS) td.bulk_cols = rows_bulk ? (td.ncols / V) * V : 0;  // whole 16-byte chunks only
         if (td.bulk_cols == 0) continue;
         const uint32_t bytes = static_cast<uint32_t>(td.bulk_cols) * sizeof(GT);
         for (int k = 0; k < N; ++k) {
@@ -511,7 +561,8 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
             timed_out = true;
             break;
           }
-          const GT* src = td.grad + static_cast<long long>(order_s[k]) * td.ld;
+          const GT* src = ROWS ? rowptr_s[k] + static_cast<long long>(tile) * TILE
+                               : td.grad + static_cast<long long>(order_s[k]) * td.ld;
           mbar_arrive_expect_tx(full_addr + 8u * s, bytes);
           bulk_copy_g2s(ring_addr + static_cast<uint32_t>(s) * STAGE_BYTES, src, bytes,
                         full_addr + 8u * s, policy);
@@ -528,7 +579,11 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
     int s = 0;
     uint32_t phase = 0;
     for (int tile = blockIdx.x; tile < total_tiles && !timed_out; tile += gridDim.x) {
-      const TileDesc<GT> td = locate_tile<GT, TILE, EP>(p, prefix_s, tile);
+      TileDesc<GT> td = locate_tile<GT, TILE, EP>(p, prefix_s, tile);
+      if constexpr (ROWS) {
+        td.bulk_cols = rows_bulk ? (td.ncols / V) * V : 0;
+        td.vec_ok = td.vec_ok && repl_vec;
+      }
 
       float acc[CH][V];
 #pragma unroll
@@ -539,7 +594,8 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
       // columns of this thread that the bulk copy did not deliver (ragged end, unaligned
       // segment) are read straight from global memory, row by row, in the same order
       auto add_row_tail = [&](int k) {
-        const GT* row = td.grad + static_cast<long long>(order_s[k]) * td.ld;
+        const GT* row = ROWS ? rowptr_s[k] + static_cast<long long>(tile) * TILE
+                             : td.grad + static_cast<long long>(order_s[k]) * td.ld;
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
           const int o = (tid + c * NT) * V;
@@ -696,6 +752,10 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
             store_floats<V>(td.theta + o, vec, n, th);
             if (Rule::kState0) store_floats<V>(td.s0 + o, vec, n, s0);
             if (Rule::kState1) store_floats<V>(td.s1 + o, vec, n, s1);
+            if constexpr (ROWS) {  // the workers' copies of this shard
+              for (int r = 0; r < p.R; ++r)
+                store_floats<V>(repl_s[r] + static_cast<long long>(tile) * TILE + o, vec, n, th);
+            }
           }
         }
       }
