@@ -473,6 +473,42 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
             assert info3.cpu().tolist() == [m_all, 0, 4 * m_kept]
             out["two_level"] = dict(rates(4 * m_kept * P * esize + state_bytes, 4 * m_kept * P * esize, ms),
                                     machines=m_all, machines_kept=m_kept, rows_used=4 * m_kept)
+        # the step as parameter servers run it (rows given by address): one server owning every column, then
+        # eight servers over eight ranges, each pushing its new parameters into the seven other copies of theta --
+        # the launches of an 8-GPU job, run one after another on this one GPU
+        rows_all = sgdb.make_address_table([grad[w].data_ptr() for w in range(W)], dev)
+
+        def rows_step(i):
+            opt.step = i + 1
+            sgdb.sgdb_step_rows(rows_all, grad.dtype, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, None,
+                                mask, order, info)
+
+        ms = time_steps(rows_step, 20, 3)
+        out["rows_by_address"] = rates(N * P * esize + state_bytes, N * P * esize, ms)
+        G = 8
+        free, _ = torch.cuda.mem_get_info(dev)
+        if free > (G + 2) * P * 4 + (1 << 30):
+            copies = [theta] + [theta.clone() for _ in range(G - 1)]
+            ranges = [sgdb.sgdb_shard_range(P, G, j) for j in range(G)]
+            row_tables = [sgdb.make_address_table([grad[w].data_ptr() + first * esize for w in range(W)], dev)
+                          for first, _ in ranges]
+            push_tables = [sgdb.make_address_table([copies[g].data_ptr() + first * 4 for g in range(G) if g != j], dev)
+                           for j, (first, _) in enumerate(ranges)]
+            cut = lambda x, first, n: None if x is None else x[first:first + n]
+
+            def servers_step(i):
+                opt.step = i + 1
+                for j, (first, n) in enumerate(ranges):
+                    sgdb.sgdb_step_rows(row_tables[j], grad.dtype, n, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b,
+                                        cut(copies[j], first, n), cut(s0, first, n), cut(s1, first, n), opt, push_tables[j],
+                                        mask, order, info)
+
+            ms = time_steps(servers_step, 20, 3)
+            assert all(torch.equal(c, copies[0]) for c in copies[1:]), "the copies of theta differ"
+            pushed = (G - 1) * P * 4
+            out["eight_servers_on_one_gpu"] = dict(rates(N * P * esize + state_bytes + pushed, N * P * esize, ms), servers=G,
+                                                   launches_per_step=G, pushed_bytes_per_step=pushed)
+            del copies, row_tables, push_tables
         assert info.cpu().tolist()[1] == 0 and bool(torch.isfinite(theta).all())
         return out
 
@@ -768,6 +804,87 @@ def run_native(args, cfg):
     finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks, cpu)
 
 
+def run_servers(args, cfg):
+    """The several-GPUs form, one process per parameter server (`--servers`): the workers' gradient rows are whole
+    rows spread over the GPUs' memories, GPU j updates its range of columns in one launch that pulls the kept rows
+    from wherever they live and pushes the new parameters into every GPU's copy.  P is the whole model whatever the
+    number of GPUs (strong scaling); what bounds it beyond one GPU is the link, not HBM."""
+    import torch.distributed as dist
+
+    from paper_1604_00981_b200 import binding as sgdb
+    from paper_1604_00981_b200 import servers
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29531")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
+    tdt = torch.float32 if cfg.grad_dtype == "f32" else torch.bfloat16
+    srv = servers.ServerGroup(P, W, N, b, tdt, cfg.opt, dev)
+    mine = srv.plan.workers_of(rank)
+    scales = wl.worker_scales(cfg.seed, W)
+    if len(mine):
+        wl.grad_matrix(cfg.seed + 1000 * rank, 0, len(mine), P, scales[mine.start:mine.stop], cfg.grad_dtype, dev,
+                       ld=srv.grads.stride(0), out=srv.grads[:len(mine)])
+    srv.theta[:P] = wl.theta0(cfg.seed, P, dev)
+    arr_d, tag_d = selection_sets(cfg, dev)
+
+    def step(i):
+        srv.step(0, arr_d[i % N_SETS], tag_d[i % N_SETS], update=i + 1)
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        start.record()
+        for i in range(args.steps):
+            step(args.warmup + i)
+        stop.record()
+        barrier()
+    ms_total = max_over_ranks(dist, [start.elapsed_time(stop)], dev)[0]
+    assert srv.info[:2].cpu().tolist()[1] == 0 and bool(torch.isfinite(srv.theta).all())
+    if rank == 0:
+        esize = 4 if cfg.grad_dtype == "f32" else 2
+        ms = ms_total / args.steps
+        grad_bytes = N * P * esize
+        first, n = srv.plan.ranges[0]
+        # per GPU and step: its columns of the kept rows, theta and state of its range read and written, its range
+        # stored into the other copies; of the rows, (G - 1) / G arrive over the link on average
+        per_gpu = N * n * esize + 2 * (1 + N_STATE[cfg.opt["kind"]]) * n * 4 + (world - 1) * n * 4
+        link = N * n * esize * (world - 1) / world
+        hbm_peak, peak_kind = measured_hbm_peak()
+        if world == 1:
+            roof = {"bound": "hbm", "achieved": per_gpu / (ms * 1e-3) / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                    "peak_source": peak_kind}
+        else:
+            roof = {"bound": "nvlink", "achieved": link / (ms * 1e-3) / 1e9, "peak": 770.0, "unit": "GB/s",
+                    "peak_source": "peer copy measured on this pool, per direction"}
+        roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": None,
+                     "kernel": "stream_rows_kernel<%s, %s, rows by address>, one launch per GPU and step" % (cfg.grad_dtype, cfg.opt["kind"]),
+                     "algorithmic_bytes_per_step": per_gpu, "link_bytes_per_step": link})
+        config = workload_config(cfg, P, grad_bytes, grad_bytes + 2 * (1 + N_STATE[cfg.opt["kind"]]) * P * 4)
+        config["sharding"] = ("%d parameter servers, one per GPU: columns split in %d ranges, workers' rows spread over the "
+                              "GPUs, no collective (pull + push inside the one launch, fences between)" % (world, world))
+        print(json.dumps({
+            "metric": METRIC, "value": grad_bytes / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": cfg.grad_dtype, "data": "synthetic", "config": config, "step_us": ms * 1e3, "roofline": roof,
+            "e2e": None, "gpu_launches": args.steps, "clocks": clocks.summary(), "cpu_baseline": None}), flush=True)
+    dist.destroy_process_group()
+
+
 def finish(args, cfg, wk, extra, dist, dev, rank, world, ms_total, e2e_ms, e2e_steps, clocks, cpu):
     W, N, b = cfg.W, cfg.N, cfg.b
     P = wk.get("P", cfg.P)
@@ -832,6 +949,10 @@ def main():
                     help="flat workloads: time-out rule (sgdb_step_deadline) with this deadline in seconds")
     ap.add_argument("--machines", type=int, default=0,
                     help="flat workloads: two-level aggregation (sgdb_step_grouped) with the workers spread over this many machines")
+    ap.add_argument("--servers", action="store_true",
+                    help="flat workloads: one process per parameter server over the WHOLE model (rows pulled from and "
+                         "parameters pushed to the other GPUs inside the one launch); default is one independent column "
+                         "shard per GPU")
     ap.add_argument("--columns", type=int, default=0,
                     help="override P with a smaller column count (profiler captures); not the benchmark workload")
     ap.add_argument("--rows", type=int, default=0,
@@ -853,6 +974,8 @@ def main():
         cfg = dataclasses.replace(cfg, N=args.rows, name=cfg.name + "_rows_%d" % args.rows)
     if args.impl == "reference":
         run_reference(args, cfg)
+    elif args.servers:
+        run_servers(args, cfg)
     else:
         run_native(args, cfg)
 

@@ -84,6 +84,8 @@ def share_with_peers(tensor: torch.Tensor, group=None):
     shared-memory file; the owner must keep its tensor alive while the peers use theirs."""
     world = dist.get_world_size(group)
     rank = dist.get_rank(group)
+    if world == 1:
+        return [tensor]
     payload = bytes(ForkingPickler.dumps(tensor))
     gathered = [None] * world
     dist.all_gather_object(gathered, payload, group=group)
