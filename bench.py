@@ -49,7 +49,7 @@ NOMINAL_HBM_GBS = 8000.0
 
 # DRAM traffic of one fused-step launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
 # as bytes per algorithmic byte; valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"src_digest": "4208c3027d17c36b", "dram_bytes_per_algorithmic_byte": 0.9956}
+NCU_TRAFFIC = {"src_digest": "34567afc489004ab", "dram_bytes_per_algorithmic_byte": 0.9956}
 
 
 def kernel_source_digest() -> str:
@@ -823,7 +823,10 @@ def run_servers(args, cfg):
     os.environ.setdefault("MASTER_PORT", "29531")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    if world > 1:
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    else:  # a group of one needs no device collective: nothing crosses, the fences have nobody to wait for
+        dist.init_process_group("gloo", rank=0, world_size=1)
     W, N, b, P = cfg.W, cfg.N, cfg.b, cfg.P
     tdt = torch.float32 if cfg.grad_dtype == "f32" else torch.bfloat16
     srv = servers.ServerGroup(P, W, N, b, tdt, cfg.opt, dev)
@@ -839,7 +842,8 @@ def run_servers(args, cfg):
         srv.step(0, arr_d[i % N_SETS], tag_d[i % N_SETS], update=i + 1)
 
     def barrier():
-        dist.barrier()
+        if world > 1:
+            dist.barrier()
         torch.cuda.synchronize()
 
     for i in range(args.warmup):
@@ -853,7 +857,7 @@ def run_servers(args, cfg):
             step(args.warmup + i)
         stop.record()
         barrier()
-    ms_total = max_over_ranks(dist, [start.elapsed_time(stop)], dev)[0]
+    ms_total = max_over_ranks(dist if world > 1 else None, [start.elapsed_time(stop)], dev)[0]
     assert srv.info[:2].cpu().tolist()[1] == 0 and bool(torch.isfinite(srv.theta).all())
     if rank == 0:
         esize = 4 if cfg.grad_dtype == "f32" else 2

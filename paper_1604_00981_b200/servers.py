@@ -96,6 +96,8 @@ def fence(group=None, flag: torch.Tensor | None = None) -> None:
     """Everything enqueued before the fence on any rank's current stream is complete, on every rank, before
     anything enqueued after it starts.  With NCCL this is a one-word all-reduce on the stream (no host wait);
     with another backend the host waits for its stream and meets the others at a barrier."""
+    if dist.get_world_size(group) == 1:
+        return  # the stream's own order is all there is to keep
     backend = dist.get_backend(group)
     if backend == "nccl":
         dist.all_reduce(flag, group=group)
