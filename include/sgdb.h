@@ -510,6 +510,17 @@ sgdb_status_t sgdb_set_tuning(int32_t stages, int32_t ctas_per_sm);
  */
 sgdb_status_t sgdb_set_arrival_tuning(int64_t resident_bytes, int32_t blocks_per_sm);
 
+/*
+ * sgdb_selftest_bounded_wait -- shows on the device that a wait inside the kernels cannot hang (no
+ * counterpart in the paper).  Every on-chip wait of the row-streaming kernels is bounded by wall time and
+ * ends in SGDB_ERR_TIMEOUT; in a correct run that never happens, so this call exercises the same wait
+ * routine on a barrier that nothing will ever complete: one small block waits for `limit_ns`
+ * (0 .. 100 ms, larger values are refused), gives up, and the kernel ends normally.
+ *   d_out [3] int32 out: {SGDB_ERR_TIMEOUT, nanoseconds waited, 1 if a second waiter was released by the
+ *                         first one's give-up}
+ */
+sgdb_status_t sgdb_selftest_bounded_wait(int64_t limit_ns, int32_t *d_out, void *stream);
+
 const char *sgdb_strerror(sgdb_status_t status); /* static string, never NULL */
 int sgdb_version(void);                          /* major*10000 + minor*100 + patch */
 

@@ -28,7 +28,7 @@ EXPORTS = (
     "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_accumulate_arrival_ema", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
     "sgdb_select_grouped", "sgdb_step_grouped", "sgdb_step_segmented_ema", "sgdb_step_segmented_deadline",
     "sgdb_accumulate_arrival_deadline", "sgdb_accumulate_close", "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version",
-    "sgdb_step_rows", "sgdb_step_rows_ordered", "sgdb_shard_range",
+    "sgdb_step_rows", "sgdb_step_rows_ordered", "sgdb_shard_range", "sgdb_selftest_bounded_wait",
 )
 SGDB_STATIC_SCRATCH_BYTES = 8 << 20
 SGDB_MAX_REPLICAS = 64
@@ -119,6 +119,7 @@ def _load():
         "sgdb_step_host_workspace_bytes": (sz, [i32, i64, i64, i32, i32]),
         "sgdb_step_host_static": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt),
                                         vp, vp, vp, vp, vp]),
+        "sgdb_selftest_bounded_wait": (i32, [i64, vp, vp]),
         "sgdb_set_tuning": (i32, [i32, i32]),
         "sgdb_set_arrival_tuning": (i32, [i64, i32]),
         "sgdb_strerror": (ctypes.c_char_p, [i32]),
@@ -178,6 +179,13 @@ def sgdb_strerror(status: int) -> str:
 
 def sgdb_version() -> int:
     return int(_lib.sgdb_version())
+
+
+def sgdb_selftest_bounded_wait(limit_ns: int, out, stream=None) -> None:
+    """A wait for a barrier that nothing completes, with the kernels' own wait routine: out i32[3] receives
+    {SGDB_ERR_TIMEOUT, nanoseconds waited, 1 if a second waiter was released by the give-up}."""
+    _check(_lib.sgdb_selftest_bounded_wait(limit_ns, _dev(out, torch.int32, "out"), _stream(stream)),
+           "sgdb_selftest_bounded_wait")
 
 
 def sgdb_set_tuning(stages: int = 0, ctas_per_sm: int = 0) -> None:

@@ -930,6 +930,13 @@ sgdb_status_t sgdb_set_arrival_tuning(int64_t resident_bytes, int32_t blocks_per
   return SGDB_OK;
 }
 
+sgdb_status_t sgdb_selftest_bounded_wait(int64_t limit_ns, int32_t* d_out, void* stream) {
+  if (d_out == nullptr || limit_ns < 0 || limit_ns > 100ll * 1000 * 1000) return SGDB_ERR_INVALID_ARG;
+  bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<unsigned long long>(limit_ns),
+                                                                                d_out);
+  return launch_status();
+}
+
 const char* sgdb_strerror(sgdb_status_t status) {
   switch (status) {
     case SGDB_OK: return "ok";

@@ -1095,4 +1095,34 @@ __global__ void __launch_bounds__(256, 4) close_iteration_kernel(const ClosePara
   }
 }
 
+// ====================================================================== bounded wait, on its own
+//
+// One block arms nothing and waits, with the same routine the row-streaming kernel uses, for a barrier
+// phase that nobody will ever complete.  The wait must give up after `limit_ns`, raise the block's abort
+// flag and let the kernel end normally; the second warp, which watches only the flag, must see it.
+//   out[0] = SGDB_ERR_TIMEOUT when the wait gave up (SGDB_OK if it claims the phase completed)
+//   out[1] = nanoseconds the waiting thread spent, clamped to int32
+//   out[2] = 1 when the watching warp left through the abort flag
+__global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(unsigned long long limit_ns, int32_t* out) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int s_abort;
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    mbar_init(smem_addr(&bar), 1);
+    fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned long long t0 = global_timer_ns();
+    const bool done = mbar_wait_for(smem_addr(&bar), 0u, &s_abort, limit_ns);
+    const unsigned long long waited = global_timer_ns() - t0;
+    out[0] = done ? SGDB_OK : SGDB_ERR_TIMEOUT;
+    out[1] = waited > 0x7fffffffull ? 0x7fffffff : static_cast<int32_t>(waited);
+  } else if (threadIdx.x == 32) {
+    // a second waiter with a limit it cannot reach first: it leaves because the first raised the flag
+    const bool done = mbar_wait_for(smem_addr(&bar), 0u, &s_abort, limit_ns + kWaitLimitNs);
+    out[2] = (!done && s_abort != 0) ? 1 : 0;
+  }
+}
+
 }  // namespace sgdb
