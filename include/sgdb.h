@@ -364,6 +364,15 @@ sgdb_status_t sgdb_step_rows_ordered(const void *const *d_rows, int32_t W, sgdb_
 sgdb_status_t sgdb_shard_range(int64_t P, int32_t n_servers, int32_t j, int64_t *first, int64_t *len);
 
 /*
+ * sgdb_enable_peer_access -- lets kernels launched on the CURRENT device read and write the memory of
+ * `peer_device` (what sgdb_step_rows needs before it is given a peer's addresses; no counterpart in the
+ * paper).  Enabling twice is fine; the current device itself is accepted and needs nothing.
+ * SGDB_ERR_UNSUPPORTED when the two devices have no peer path, SGDB_ERR_INVALID_ARG for a device that does
+ * not exist.  This is a one-time set-up call of the process, not part of an iteration.
+ */
+sgdb_status_t sgdb_enable_peer_access(int32_t peer_device);
+
+/*
  * sgdb_accumulate_arrival -- Algorithm 4's inner loop taken literally: one
  * gradient per call, in the order the gradients reach the server.
  *

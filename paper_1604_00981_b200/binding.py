@@ -28,7 +28,7 @@ EXPORTS = (
     "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_accumulate_arrival_ema", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
     "sgdb_select_grouped", "sgdb_step_grouped", "sgdb_step_segmented_ema", "sgdb_step_segmented_deadline",
     "sgdb_accumulate_arrival_deadline", "sgdb_accumulate_close", "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version",
-    "sgdb_step_rows", "sgdb_step_rows_ordered", "sgdb_shard_range", "sgdb_selftest_bounded_wait",
+    "sgdb_step_rows", "sgdb_step_rows_ordered", "sgdb_shard_range", "sgdb_enable_peer_access", "sgdb_selftest_bounded_wait",
 )
 SGDB_STATIC_SCRATCH_BYTES = 8 << 20
 SGDB_MAX_REPLICAS = 64
@@ -120,6 +120,7 @@ def _load():
         "sgdb_step_host_static": (i32, [vp, i32, i64, i64, vp, vp, i32, i32, i32, vp, vp, vp, ctypes.POINTER(_COpt),
                                         vp, vp, vp, vp, vp]),
         "sgdb_selftest_bounded_wait": (i32, [i64, vp, vp]),
+        "sgdb_enable_peer_access": (i32, [i32]),
         "sgdb_set_tuning": (i32, [i32, i32]),
         "sgdb_set_arrival_tuning": (i32, [i64, i32]),
         "sgdb_strerror": (ctypes.c_char_p, [i32]),
@@ -426,6 +427,11 @@ def sgdb_shard_range(P: int, n_servers: int, j: int):
     first, length = ctypes.c_int64(0), ctypes.c_int64(0)
     _check(_lib.sgdb_shard_range(P, n_servers, j, ctypes.byref(first), ctypes.byref(length)), "sgdb_shard_range")
     return int(first.value), int(length.value)
+
+
+def sgdb_enable_peer_access(peer_device: int) -> None:
+    """Kernels launched on the current device may then use the memory of peer_device (one-time set-up)."""
+    _check(_lib.sgdb_enable_peer_access(int(peer_device)), "sgdb_enable_peer_access")
 
 
 def sgdb_accumulate_arrival(row, row_tag: int, t: int, N: int, acc, counter, theta, state0, state1,

@@ -44,12 +44,13 @@ constexpr int kDefaultStages = 7;
 constexpr int kDefaultCtasPerSm = 2;
 
 struct DeviceInfo {
-  bool known = false;
+  std::atomic<bool> known{false};  // set last, with release: a reader that sees it sees the other fields
   int index = 0;
   int sms = 0;
   int max_smem_optin = 0;
 };
 DeviceInfo g_dev[kMaxDevices];
+std::mutex g_dev_mutex;
 int g_stages = kDefaultStages;
 int g_ctas_per_sm = kDefaultCtasPerSm;
 constexpr int kDefaultArrivalBlocksPerSm = 4;
@@ -66,13 +67,16 @@ sgdb_status_t device_info(const DeviceInfo** out) {
   if (cudaGetDevice(&dev) != cudaSuccess) return SGDB_ERR_CUDA;
   if (dev < 0 || dev >= kMaxDevices) return SGDB_ERR_UNSUPPORTED;
   DeviceInfo& d = g_dev[dev];
-  if (!d.known) {
-    if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) !=
-            cudaSuccess)
-      return SGDB_ERR_CUDA;
-    d.index = dev;
-    d.known = true;
+  if (!d.known.load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (!d.known.load(std::memory_order_relaxed)) {
+      if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) !=
+              cudaSuccess)
+        return SGDB_ERR_CUDA;
+      d.index = dev;
+      d.known.store(true, std::memory_order_release);
+    }
   }
   *out = &d;
   return SGDB_OK;
@@ -766,6 +770,22 @@ sgdb_status_t sgdb_step_rows_ordered(const void* const* d_rows, int32_t W, sgdb_
   p.info = d_info;
   p.status_out = d_info + 1;
   return launch_stream_rows(dt, ep, p, static_cast<cudaStream_t>(stream));
+}
+
+sgdb_status_t sgdb_enable_peer_access(int32_t peer_device) {
+  int dev = 0, count = 0, can = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceCount(&count) != cudaSuccess) return launch_status();
+  if (peer_device < 0 || peer_device >= count) return SGDB_ERR_INVALID_ARG;
+  if (peer_device == dev) return SGDB_OK;  // a device reaches its own memory as it is
+  if (cudaDeviceCanAccessPeer(&can, dev, peer_device) != cudaSuccess) return launch_status();
+  if (!can) return SGDB_ERR_UNSUPPORTED;
+  const cudaError_t e = cudaDeviceEnablePeerAccess(peer_device, 0);
+  if (e == cudaErrorPeerAccessAlreadyEnabled) {
+    (void)cudaGetLastError();
+    return SGDB_OK;
+  }
+  if (e != cudaSuccess) return launch_status();
+  return SGDB_OK;
 }
 
 sgdb_status_t sgdb_shard_range(int64_t P, int32_t n_servers, int32_t j, int64_t* first, int64_t* len) {

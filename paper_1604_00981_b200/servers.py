@@ -155,6 +155,12 @@ class ServerGroup:
         self._peer_grads = share_with_peers(self.grads, group)
         self._peer_theta = share_with_peers(self.theta, group)
         self._peer_message = share_with_peers(self.message, group)
+        if self.device.type == "cuda":
+            # kernels on this GPU will read the peers' rows and write the peers' copies of theta
+            with torch.cuda.device(self.device):
+                for x in self._peer_grads:
+                    if x.device != self.grads.device:
+                        binding.sgdb_enable_peer_access(x.device.index)
         pitch = self.grads.stride(0) * es
         self.row_addr = row_addresses(self.plan, self.rank, [x.data_ptr() for x in self._peer_grads], pitch, es)
         self.replica_addr = replica_addresses(self.plan, self.rank, [x.data_ptr() for x in self._peer_theta])

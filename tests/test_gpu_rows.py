@@ -282,3 +282,20 @@ def test_rows_mid_size_four_servers(sgdb, cuda_device):
     assert rc == oracle.OK
     assert rel_err(copies[0][cols_d].cpu().numpy(), th_o) < TOL_F32
     assert torch.equal(torch.cat([states[j][0] for j in range(G)]), s1[0])
+
+
+def test_peer_access_set_up_call(sgdb, cuda_device):
+    """The set-up call for a peer's memory: the current device itself needs nothing, a device that does not exist is
+    refused; with a second device present, enabling twice is fine."""
+    sgdb.sgdb_enable_peer_access(torch.cuda.current_device())
+    for bad in (-1, torch.cuda.device_count()):
+        with pytest.raises(sgdb.SgdbError) as e:
+            sgdb.sgdb_enable_peer_access(bad)
+        assert e.value.status == sgdb.SGDB_ERR_INVALID_ARG
+    if torch.cuda.device_count() > 1:
+        other = (torch.cuda.current_device() + 1) % torch.cuda.device_count()
+        try:
+            sgdb.sgdb_enable_peer_access(other)
+            sgdb.sgdb_enable_peer_access(other)
+        except sgdb.SgdbError as e:
+            assert e.status == sgdb.SGDB_ERR_UNSUPPORTED
