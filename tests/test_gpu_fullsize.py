@@ -403,3 +403,54 @@ def test_config2_full_size_every_element_against_the_oracle(sgdb, cuda_device):
     assert rel_err(got, want) < TOL_F32
     assert rel_err(np.concatenate([r[2] for r in results]), np.concatenate([r[3] for r in results])) < TOL_F32
     assert float(np.max(np.abs(got - want) / np.maximum(np.abs(want), 1e-2))) < 1e-4
+
+
+def test_more_columns_than_a_32_bit_index_holds(sgdb, cuda_device):
+    """P = 2^31 + 4099 columns (8.6 GB per fp32 vector), W = 3 (N = 2, b = 1), plain SGD: every column index, tile
+    start and byte offset beyond 2^31 must be computed in 64 bits.  The fused step against the oracle at sampled
+    columns (the first, the last, both sides of 2^31 and of 2^32 bytes); the separate calls, the rows-by-address
+    step and the arrival-by-arrival server against the fused step on the whole vector, bit for bit."""
+    _need_memory(cuda_device, 80)
+    dev = cuda_device
+    P, W, N, b, seed = (1 << 31) + 4099, 3, 2, 1, 977
+    opt_kw = dict(kind="sgd", lr=0.1)
+    rng = np.random.default_rng(seed)
+    edges = np.concatenate([np.arange(e - 3, e + 3) for e in ((1 << 30), (1 << 31), (1 << 31) + 2048, P - 3)])
+    cols = np.unique(np.concatenate([_sample_columns(P, rng, n=2000), edges[(edges >= 0) & (edges < P)]]))
+    cols_d = to_dev(cols, dev)
+    grad = wl.grad_matrix(seed, 0, W, P, wl.worker_scales(seed, W), "f32", dev)
+    arrival = np.array([2.0, 1.0, 3.0], np.float32)
+    tags = np.zeros(W, np.int32)
+    a_d, t_d = to_dev(arrival, dev), to_dev(tags, dev)
+    theta = wl.theta0(seed, P, dev)
+    th_o = theta[cols_d].cpu().numpy().astype(np.float64)
+    twin = theta.clone()
+    mask, order, info = selection_buffers(W, N, dev)
+    sgdb.sgdb_step(grad, P, a_d, t_d, 0, N, b, theta, None, None, gpu_opt(opt_kw), mask, order, info)
+    rc, mask_o, order_o, n_valid = oracle.step(wl.as_oracle_array(grad.index_select(1, cols_d)), len(cols), arrival, tags, 0,
+                                               N, b, th_o, None, None, oracle_opt(opt_kw))
+    assert rc == oracle.OK and info.cpu().tolist() == [n_valid, 0] and order.cpu().numpy().tolist() == order_o.tolist()
+    assert rel_err(theta[cols_d].cpu().numpy(), th_o) < TOL_F32
+    # separate calls: the mean goes through memory
+    mean = torch.empty(P, device=dev)
+    sgdb.sgdb_aggregate(grad, P, N, order, info, mean)
+    sgdb.sgdb_update(twin, None, None, mean, gpu_opt(opt_kw), info)
+    assert torch.equal(twin, theta)
+    # the arrival-by-arrival server, the running sum in the buffer that held the mean; rows in delivery sequence
+    twin.copy_(wl.theta0(seed, P, dev))
+    counter = torch.zeros(4, dtype=torch.int32, device=dev)
+    ainfo = torch.zeros(2, dtype=torch.int32, device=dev)
+    for w in wl.delivery_sequence(arrival):
+        sgdb.sgdb_accumulate_arrival(grad[w], 0, 0, N, mean, counter, twin, None, None, gpu_opt(opt_kw), ainfo)
+    assert counter.cpu().tolist() == [0, W, 0, 1] and torch.equal(twin, theta)
+    # every row at its own address, two servers over two ranges, each storing into the other's copy as well
+    del mean
+    twin.copy_(wl.theta0(seed, P, dev))
+    other = twin.clone()
+    for j, copies in ((0, (twin, other)), (1, (other, twin))):
+        first, n = sgdb.sgdb_shard_range(P, 2, j)
+        rows = sgdb.make_address_table([grad[w].data_ptr() + first * 4 for w in range(W)], dev)
+        push = sgdb.make_address_table([copies[1].data_ptr() + first * 4], dev)
+        sgdb.sgdb_step_rows(rows, torch.float32, n, a_d, t_d, 0, N, b, copies[0][first:first + n], None, None, gpu_opt(opt_kw),
+                            push, mask, order, info)
+    assert torch.equal(twin, theta) and torch.equal(other, theta)
