@@ -509,6 +509,17 @@ sgdb_status_t sgdb_step_host_static(const void *h_grad, sgdb_dtype_t dt, int64_t
 sgdb_status_t sgdb_set_tuning(int32_t stages, int32_t ctas_per_sm);
 
 /*
+ * sgdb_set_wait_limit_ns -- patience of the waits inside the row-streaming kernels (no counterpart in the
+ * paper).  Every wait of those kernels on a shared-memory barrier gives up after this many nanoseconds of wall
+ * time; the kernel then stops, waits for the copies it still has in flight, reports SGDB_ERR_TIMEOUT in
+ * d_info[1] and ends normally -- theta and state may then be updated in part and must be considered lost.
+ * Default 2 s, which no correct run comes near (a wait lasts microseconds).  A negative value restores the
+ * default; 0 means no patience at all -- a wait whose data is not there yet gives up at once, which happens
+ * in every launch (used by the tests to show on the device that the path works); values above 10 s are refused.  Affects later calls of this process.
+ */
+sgdb_status_t sgdb_set_wait_limit_ns(int64_t limit_ns);
+
+/*
  * sgdb_set_arrival_tuning -- launch-shape knobs of sgdb_accumulate_arrival (no counterpart
  * in the paper).  resident_bytes: how many leading bytes of the running sum d_acc the
  * kernels ask the L2 cache to keep between one arrival's launch and the next (the sum is

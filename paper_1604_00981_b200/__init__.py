@@ -17,7 +17,7 @@ _BINDING_NAMES = (
     "sgdb_select", "sgdb_aggregate", "sgdb_update", "sgdb_step", "sgdb_step_segmented", "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate",
     "sgdb_accumulate_arrival", "sgdb_accumulate_arrival_ema", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
     "sgdb_select_grouped", "sgdb_step_grouped", "sgdb_step_segmented_ema", "sgdb_step_segmented_deadline", "sgdb_accumulate_arrival_deadline", "sgdb_accumulate_close", "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version", "Opt", "SgdbError",
-    "sgdb_step_rows", "sgdb_step_rows_ordered", "sgdb_shard_range", "sgdb_enable_peer_access", "sgdb_selftest_bounded_wait",
+    "sgdb_step_rows", "sgdb_step_rows_ordered", "sgdb_shard_range", "sgdb_enable_peer_access", "sgdb_selftest_bounded_wait", "sgdb_set_wait_limit_ns",
     "make_address_table",
 )
 

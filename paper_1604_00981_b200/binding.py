@@ -28,7 +28,7 @@ EXPORTS = (
     "sgdb_select_deadline", "sgdb_step_deadline", "sgdb_step_ema", "sgdb_ema", "sgdb_learning_rate", "sgdb_accumulate_arrival", "sgdb_accumulate_arrival_ema", "sgdb_step_host", "sgdb_step_host_workspace_bytes", "sgdb_step_host_static",
     "sgdb_select_grouped", "sgdb_step_grouped", "sgdb_step_segmented_ema", "sgdb_step_segmented_deadline",
     "sgdb_accumulate_arrival_deadline", "sgdb_accumulate_close", "sgdb_set_tuning", "sgdb_set_arrival_tuning", "sgdb_strerror", "sgdb_version",
-    "sgdb_step_rows", "sgdb_step_rows_ordered", "sgdb_shard_range", "sgdb_enable_peer_access", "sgdb_selftest_bounded_wait",
+    "sgdb_step_rows", "sgdb_step_rows_ordered", "sgdb_shard_range", "sgdb_enable_peer_access", "sgdb_selftest_bounded_wait", "sgdb_set_wait_limit_ns",
 )
 SGDB_STATIC_SCRATCH_BYTES = 8 << 20
 SGDB_MAX_REPLICAS = 64
@@ -122,6 +122,7 @@ def _load():
         "sgdb_selftest_bounded_wait": (i32, [i64, vp, vp]),
         "sgdb_enable_peer_access": (i32, [i32]),
         "sgdb_set_tuning": (i32, [i32, i32]),
+        "sgdb_set_wait_limit_ns": (i32, [i64]),
         "sgdb_set_arrival_tuning": (i32, [i64, i32]),
         "sgdb_strerror": (ctypes.c_char_p, [i32]),
         "sgdb_version": (ctypes.c_int, []),
@@ -191,6 +192,11 @@ def sgdb_selftest_bounded_wait(limit_ns: int, out, stream=None) -> None:
 
 def sgdb_set_tuning(stages: int = 0, ctas_per_sm: int = 0) -> None:
     _check(_lib.sgdb_set_tuning(stages, ctas_per_sm), "sgdb_set_tuning")
+
+
+def sgdb_set_wait_limit_ns(limit_ns: int = -1) -> None:
+    """Patience of the waits inside the row-streaming kernels in nanoseconds (negative: the 2 s default)."""
+    _check(_lib.sgdb_set_wait_limit_ns(limit_ns), "sgdb_set_wait_limit_ns")
 
 
 def sgdb_set_arrival_tuning(resident_bytes: int = -1, blocks_per_sm: int = 0) -> None:

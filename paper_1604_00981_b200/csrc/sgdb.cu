@@ -51,6 +51,7 @@ struct DeviceInfo {
 };
 DeviceInfo g_dev[kMaxDevices];
 std::mutex g_dev_mutex;
+std::atomic<long long> g_wait_limit_ns{static_cast<long long>(kWaitLimitNs)};
 int g_stages = kDefaultStages;
 int g_ctas_per_sm = kDefaultCtasPerSm;
 constexpr int kDefaultArrivalBlocksPerSm = 4;
@@ -184,6 +185,7 @@ sgdb_status_t launch_stream_t(const StreamParams& p_in, cudaStream_t stream) {
   const size_t smem = static_cast<size_t>(stages) * (kStageBytes + 16) + fixed;
   if (smem > per_sm_budget) return SGDB_ERR_UNSUPPORTED;
   p.stages = stages;
+  p.wait_limit_ns = static_cast<unsigned long long>(g_wait_limit_ns.load(std::memory_order_relaxed));
   // the opt-in to large dynamic shared memory is kept per kernel and device: asked for again only when a
   // launch needs more than any launch of this kernel before it
   static std::atomic<int> smem_allowed[kMaxDevices];
@@ -940,6 +942,12 @@ sgdb_status_t sgdb_set_tuning(int32_t stages, int32_t ctas_per_sm) {
   if (stages > 64 || ctas_per_sm > 8) return SGDB_ERR_INVALID_ARG;
   g_stages = stages > 0 ? (stages < 2 ? 2 : stages) : kDefaultStages;
   g_ctas_per_sm = ctas_per_sm > 0 ? ctas_per_sm : kDefaultCtasPerSm;
+  return SGDB_OK;
+}
+
+sgdb_status_t sgdb_set_wait_limit_ns(int64_t limit_ns) {
+  if (limit_ns > 10ll * 1000 * 1000 * 1000) return SGDB_ERR_INVALID_ARG;
+  g_wait_limit_ns.store(limit_ns >= 0 ? limit_ns : static_cast<long long>(kWaitLimitNs), std::memory_order_relaxed);
   return SGDB_OK;
 }
 

@@ -56,11 +56,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return done != 0;
 }
 
+// Non-blocking probe of a barrier phase (try_wait above may itself hold the thread for a while).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n"
+      "  .reg .pred p;\n"
+      "  mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "  selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+
 // Every wait on a barrier is bounded by wall time.  In a correct run a phase completes
 // within microseconds; the limit only exists so that a broken pipeline ends the kernel
 // with an error status instead of hanging the device.  `abort_flag` (shared memory)
 // lets one thread's time-out end every other thread's wait quickly.
-constexpr unsigned long long kWaitLimitNs = 2000ull * 1000 * 1000;  // 2 s
+constexpr unsigned long long kWaitLimitNs = 2000ull * 1000 * 1000;  // 2 s: the default patience
 
 __device__ __forceinline__ unsigned long long global_timer_ns() {
   unsigned long long t;
@@ -68,8 +83,14 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   return t;
 }
 
+// A limit of zero means no patience at all: the phase must be complete already, one probe decides.
 __device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                               unsigned long long limit_ns) {
+  if (limit_ns == 0ull) {
+    if (mbar_test_wait(bar, parity)) return true;
+    *abort_flag = 1;
+    return false;
+  }
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long deadline = global_timer_ns() + limit_ns;
   for (uint32_t spin = 0;; ++spin) {
@@ -83,9 +104,6 @@ __device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, vol
   return false;
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  return mbar_wait_for(bar, parity, abort_flag, kWaitLimitNs);
-}
 
 // ---------------------------------------------------------------- bulk copy global -> shared
 

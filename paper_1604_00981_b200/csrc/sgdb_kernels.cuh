@@ -334,6 +334,7 @@ struct StreamParams {
   int32_t W_rows;
   float* const* replicas;
   int32_t R;
+  unsigned long long wait_limit_ns;  // patience of every wait on a ring barrier (see mbar_wait_for)
   Hyper h;
 };
 
@@ -431,6 +432,8 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ int s_abort;
   __shared__ int s_count;
+  __shared__ unsigned s_issued;      // copies the producer has issued so far (read only after a wait ran out)
+  __shared__ int s_producer_done;    // the producer has left its loop and issues nothing more
 
   const int tid = threadIdx.x;
   const int lane = tid & 31;
@@ -503,6 +506,8 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
   }
   if (tid == 0) {
     s_abort = 0;
+    s_issued = 0u;
+    s_producer_done = 0;
     for (int s = 0; s < stages; ++s) {
       mbar_init(smem_addr(full_bar + s), 1);
       mbar_init(smem_addr(empty_bar + s), NW);
@@ -551,13 +556,14 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
       const uint64_t policy = l2_policy_evict_first();  // rows are read exactly once
       int s = 0;
       uint32_t phase = 0;
+      unsigned issued = 0u;
       for (int tile = blockIdx.x; tile < total_tiles && !timed_out; tile += gridDim.x) {
         TileDesc<GT> td = locate_tile<GT, TILE, EP>(p, prefix_s, tile);
         if constexpr (ROWS) td.bulk_cols = rows_bulk ? (td.ncols / V) * V : 0;  // whole 16-byte chunks only
         if (td.bulk_cols == 0) continue;
         const uint32_t bytes = static_cast<uint32_t>(td.bulk_cols) * sizeof(GT);
         for (int k = 0; k < N; ++k) {
-          if (!mbar_wait(empty_addr + 8u * s, phase ^ 1u, &s_abort)) {
+          if (!mbar_wait_for(empty_addr + 8u * s, phase ^ 1u, &s_abort, p.wait_limit_ns)) {
             timed_out = true;
             break;
           }
@@ -566,12 +572,17 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
           mbar_arrive_expect_tx(full_addr + 8u * s, bytes);
           bulk_copy_g2s(ring_addr + static_cast<uint32_t>(s) * STAGE_BYTES, src, bytes,
                         full_addr + 8u * s, policy);
+          ++issued;
           if (++s == stages) {
             s = 0;
             phase ^= 1u;
           }
         }
       }
+      // what a consumer needs to know if it has to wait for copies still in flight after a wait ran out
+      *reinterpret_cast<volatile unsigned*>(&s_issued) = issued;
+      __threadfence_block();
+      *reinterpret_cast<volatile int*>(&s_producer_done) = 1;
     }
   } else {
     // ------------------------------------------------------------ consumers
@@ -630,7 +641,9 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
             s = 0;
             phase ^= 1u;
           }
-          if (!mbar_wait(full_addr + 8u * sa, pa, &s_abort) || !mbar_wait(full_addr + 8u * sb, pb, &s_abort)) return false;
+          if (!mbar_wait_for(full_addr + 8u * sa, pa, &s_abort, p.wait_limit_ns) ||
+              !mbar_wait_for(full_addr + 8u * sb, pb, &s_abort, p.wait_limit_ns))
+            return false;
           const unsigned char* stage_a = smem + static_cast<size_t>(sa) * STAGE_BYTES;
           const unsigned char* stage_b = smem + static_cast<size_t>(sb) * STAGE_BYTES;
           uint4 va[CH], vb[CH];
@@ -666,7 +679,7 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
           }
         }
         if (k < k_end) {  // an odd count: the last row on its own
-          if (!mbar_wait(full_addr + 8u * s, phase, &s_abort)) return false;
+          if (!mbar_wait_for(full_addr + 8u * s, phase, &s_abort, p.wait_limit_ns)) return false;
           const unsigned char* stage = smem + static_cast<size_t>(s) * STAGE_BYTES;
 #pragma unroll
           for (int c = 0; c < CH; ++c) {
@@ -762,6 +775,25 @@ __global__ void __launch_bounds__(NT + 32, 2) stream_rows_kernel(const StreamPar
     }
   }
   if (timed_out && p.status_out != nullptr) *p.status_out = SGDB_ERR_TIMEOUT;
+  // A wait ran out somewhere in this block.  Copies the producer has issued may still be on their way into this
+  // block's shared memory, which the next block on this SM will own: thread 0 stays until they have landed.  The
+  // producer stops at its next wait (it sees the abort flag) and then publishes how many copies it issued; the
+  // most recent copy into each ring slot is the one whose barrier phase may still be open.  These waits have a
+  // patience of their own: the copies were issued to valid addresses and land within microseconds.
+  if (tid == 0 && *reinterpret_cast<volatile int*>(&s_abort) != 0) {
+    const unsigned long long give_up = global_timer_ns() + kWaitLimitNs;
+    while (*reinterpret_cast<volatile int*>(&s_producer_done) == 0 && global_timer_ns() < give_up) {
+    }
+    __threadfence_block();
+    const unsigned issued = *reinterpret_cast<volatile unsigned*>(&s_issued);
+    const unsigned first = issued > static_cast<unsigned>(stages) ? issued - static_cast<unsigned>(stages) : 0u;
+    for (unsigned i = first; i < issued; ++i) {
+      const uint32_t bar = full_addr + 8u * (i % static_cast<unsigned>(stages));
+      const uint32_t parity = (i / static_cast<unsigned>(stages)) & 1u;
+      while (!mbar_try_wait(bar, parity) && global_timer_ns() < give_up) {
+      }
+    }
+  }
 }
 
 // ====================================================================== update from a mean

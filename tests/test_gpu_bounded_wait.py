@@ -47,3 +47,44 @@ def test_a_wait_that_nothing_completes_gives_up_and_reports_it(sgdb, cuda_device
     mask, order, info = selection_buffers(W, N, dev)
     sgdb.sgdb_step(grad, P, arrival, tags, 0, N, W - N, theta, None, None, gpu_opt(OPTS["sgd"]), mask, order, info)
     assert info.cpu().tolist() == [W, 0] and torch.equal(theta, torch.full((P,), -0.1, device=dev))
+
+
+def test_the_step_gives_up_cleanly_when_its_waits_have_no_patience(sgdb, cuda_device):
+    """The product kernel itself with a patience of zero: the first wait whose data is not there yet gives up, the
+    block waits for the copies it still has in flight and the kernel ends normally with SGDB_ERR_TIMEOUT.  Nothing
+    is broken on purpose: every copy goes to a valid address and lands.  Afterwards, with the default patience back,
+    the same step gives the bits it always gives: no later block found stray bytes in its shared memory."""
+    dev = cuda_device
+    W, N, P = 12, 10, 1_500_000
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(5)
+    grad = torch.randn((W, P), device=dev, generator=gen)
+    arrival = torch.arange(1, W + 1, dtype=torch.float32, device=dev)
+    tags = torch.zeros(W, dtype=torch.int32, device=dev)
+    opt = gpu_opt(OPTS["rmsprop"])
+
+    def run():
+        theta = torch.zeros(P, device=dev)
+        s0, s1 = torch.zeros(P, device=dev), torch.zeros(P, device=dev)
+        mask, order, info = selection_buffers(W, N, dev)
+        sgdb.sgdb_step(grad, P, arrival, tags, 0, N, W - N, theta, s0, s1, opt, mask, order, info)
+        torch.cuda.synchronize()
+        return theta, s0, s1, info.cpu().tolist()
+
+    want = run()
+    assert want[3] == [W, 0]
+    gave_up = 0
+    try:
+        sgdb.sgdb_set_wait_limit_ns(0)
+        for _ in range(5):
+            status = run()[3][1]
+            gave_up += status == sgdb.SGDB_ERR_TIMEOUT
+    finally:
+        sgdb.sgdb_set_wait_limit_ns(-1)
+    assert gave_up == 5, "with no patience every launch meets a wait whose data is not there yet"
+    for _ in range(3):
+        got = run()
+        assert got[3] == [W, 0]
+        assert torch.equal(got[0], want[0]) and torch.equal(got[1], want[1]) and torch.equal(got[2], want[2])
+    with pytest.raises(sgdb.SgdbError):
+        sgdb.sgdb_set_wait_limit_ns(11_000_000_000)
