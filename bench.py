@@ -49,7 +49,7 @@ NOMINAL_HBM_GBS = 8000.0
 
 # DRAM traffic of one fused-step launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
 # as bytes per algorithmic byte; valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"src_digest": "21dcb2f0511bdbba", "dram_bytes_per_algorithmic_byte": 0.9954}
+NCU_TRAFFIC = {"src_digest": "d3cf9f22412bc48f", "dram_bytes_per_algorithmic_byte": 0.9946}
 
 
 def kernel_source_digest() -> str:
