@@ -508,6 +508,43 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
             pushed = (G - 1) * P * 4
             out["eight_servers_on_one_gpu"] = dict(rates(N * P * esize + state_bytes + pushed, N * P * esize, ms), servers=G,
                                                    launches_per_step=G, pushed_bytes_per_step=pushed)
+            # the same eight GPUs with two-level aggregation: each machine first writes the mean of its own workers'
+            # rows (all eight do, none knows yet whether its message will be used), then every server takes the
+            # first seven messages as rows; 32 small launches per step on this one GPU
+            M, m_kept, per = G, G - 1, -(-W // G)
+            bounds = [(min(W, m * per), min(W, (m + 1) * per)) for m in range(M)]
+            if all(hi > lo for lo, hi in bounds) and free > (2 * G + 2) * P * 4 + (1 << 30):
+                messages = torch.empty((M, P), device=dev)
+                message_tables = [sgdb.make_address_table([messages[m].data_ptr() + first * 4 for m in range(M)], dev)
+                                  for first, _ in ranges]
+                group = torch.from_numpy(np.repeat(np.arange(M), per)[:W].astype(np.int32)).to(dev)
+                current = torch.zeros(W, dtype=torch.int32, device=dev)
+                l_mask = torch.zeros(per, dtype=torch.uint8, device=dev)
+                l_order = torch.zeros(per, dtype=torch.int32, device=dev)
+                l_info = torch.zeros(2, dtype=torch.int32, device=dev)
+                g_order = torch.zeros(m_kept, dtype=torch.int32, device=dev)
+                g_info = torch.zeros(3, dtype=torch.int32, device=dev)
+
+                def machines_step(i):
+                    opt.step = i + 1
+                    arr = arr_d[i % N_SETS]
+                    for m, (lo, hi) in enumerate(bounds):
+                        sgdb.sgdb_select(arr[lo:hi], current[lo:hi], 0, hi - lo, 0, l_mask, l_order, l_info)
+                        sgdb.sgdb_aggregate(grad[lo:hi], P, hi - lo, l_order, l_info, messages[m])
+                    for j, (first, n) in enumerate(ranges):
+                        sgdb.sgdb_select_grouped(arr, current, group, 0, M, m_kept, mask, g_order, order_w, g_info)
+                        sgdb.sgdb_step_rows_ordered(message_tables[j], torch.float32, n, m_kept, g_order, g_info,
+                                                    cut(copies[j], first, n), cut(s0, first, n), cut(s1, first, n), opt,
+                                                    push_tables[j])
+
+                ms = time_steps(machines_step, 20, 3)
+                assert g_info.cpu().tolist()[:2] == [M, 0]
+                assert all(torch.equal(c, copies[0]) for c in copies[1:]), "the copies of theta differ"
+                moved = W * P * esize + M * P * 4 + m_kept * P * 4 + state_bytes + pushed
+                out["eight_machines_two_level_on_one_gpu"] = dict(
+                    rates(moved, W * P * esize, ms), machines=M, machines_kept=m_kept, launches_per_step=4 * G,
+                    rows_crossing_between_gpus_per_step=m_kept, pushed_bytes_per_step=pushed)
+                del messages, message_tables
             del copies, row_tables, push_tables
         assert info.cpu().tolist()[1] == 0 and bool(torch.isfinite(theta).all())
         return out
