@@ -42,7 +42,9 @@ def cpu_servers(rank: int, world: int, port: int, P: int, W: int, N: int, T: int
 
     def stand_in(server, t, arrival, tags, update):
         n = server.len
-        rows = np.stack([_f32_at(a, n) for a in server.row_addr]) if n else np.zeros((W, 0), np.float32)
+        if n == 0:  # a server without columns has nothing to pull, update or push
+            return
+        rows = np.stack([_f32_at(a, n) for a in server.row_addr])
         rc, *_ = oracle.step(np.ascontiguousarray(rows), n, arrival.numpy(), tags.numpy(), t, N, b, server.master,
                              server.master_s0, server.master_s1, oracle_opt(OPTS[kind], update))
         assert rc == oracle.OK

@@ -14,7 +14,8 @@ def _free_port() -> int:
         return s.getsockname()[1]
 
 
-@pytest.mark.parametrize("P,W,N,kind,dtype", [(300_007, 22, 18, "rmsprop", "f32"), (100_003, 9, 8, "adam", "bf16")])
+@pytest.mark.parametrize("P,W,N,kind,dtype", [(300_007, 22, 18, "rmsprop", "f32"), (100_003, 9, 8, "adam", "bf16"),
+                                              (64, 5, 4, "sgd", "f32")])  # the last: the second server has no columns
 def test_two_servers_as_two_processes_on_one_gpu(cuda_device, P, W, N, kind, dtype):
     import torch.multiprocessing as mp
 

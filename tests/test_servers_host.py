@@ -66,12 +66,14 @@ def test_addresses_point_at_the_first_column_of_each_range():
             assert (c[first:first + n] == j + 1).all()
 
 
-@pytest.mark.parametrize("P,W,N,kind", [(5000, 7, 5, "rmsprop"), (333, 4, 4, "adam")])
-def test_two_servers_as_two_gloo_ranks(P, W, N, kind):
-    """Two processes, two parameter servers: after every iteration each process's copy of theta equals the
+@pytest.mark.parametrize("G,P,W,N,kind", [(2, 5000, 7, 5, "rmsprop"), (2, 333, 4, 4, "adam"), (3, 1000, 7, 6, "momentum"),
+                                          (3, 100, 5, 4, "sgd"), (4, 777, 3, 2, "adagrad")])
+def test_servers_as_gloo_ranks(G, P, W, N, kind):
+    """G processes, G parameter servers (uneven numbers of workers per machine, a machine without workers, a
+    server without columns among the cases): after every iteration each process's copy of theta equals the
     iteration computed in one piece."""
     import torch.multiprocessing as mp
 
     import servers_child
 
-    mp.spawn(servers_child.cpu_servers, args=(2, _free_port(), P, W, N, 3, kind), nprocs=2, join=True)
+    mp.spawn(servers_child.cpu_servers, args=(G, _free_port(), P, W, N, 3, kind), nprocs=G, join=True)
