@@ -299,3 +299,31 @@ def test_peer_access_set_up_call(sgdb, cuda_device):
             sgdb.sgdb_enable_peer_access(other)
         except sgdb.SgdbError as e:
             assert e.status == sgdb.SGDB_ERR_UNSUPPORTED
+
+
+def test_rows_at_the_largest_counts(sgdb, cuda_device):
+    """As many workers and as many copies of theta as the library accepts: W = 1024 rows by address (N = 1000 kept),
+    64 replicas; the bits of sgdb_step in theta and in every replica."""
+    dev = cuda_device
+    W, N, P, R, seed = sgdb.SGDB_MAX_WORKERS, 1000, 6000, sgdb.SGDB_MAX_REPLICAS, 233
+    grad = wl.grad_matrix(seed, 0, W, P, wl.worker_scales(seed, W), "f32", dev)
+    arrival = wl.arrivals(seed, 0, W)
+    arrival[: W // 8] = arrival[W // 8: 2 * (W // 8)]  # plenty of equal times
+    tags = np.zeros(W, np.int32)
+    tags[np.random.default_rng(seed).choice(W, size=10, replace=False)] = -1  # ten stragglers of the previous iteration
+    a_d, t_d = to_dev(arrival, dev), to_dev(tags, dev)
+    theta_1 = wl.theta0(seed, P, dev)
+    theta = theta_1.clone()
+    s1, s = gpu_state("adam", P, dev), gpu_state("adam", P, dev)
+    mask_1, order_1, info_1 = selection_buffers(W, N, dev)
+    sgdb.sgdb_step(grad, P, a_d, t_d, 0, N, W - N, theta_1, s1[0], s1[1], gpu_opt(OPTS["adam"]), mask_1, order_1, info_1)
+    copies = torch.zeros((R, P), device=dev)
+    rows = sgdb.make_address_table([grad[w].data_ptr() for w in range(W)], dev)
+    push = sgdb.make_address_table([copies[r].data_ptr() for r in range(R)], dev)
+    mask, order, info = selection_buffers(W, N, dev)
+    sgdb.sgdb_step_rows(rows, torch.float32, P, a_d, t_d, 0, N, W - N, theta, s[0], s[1], gpu_opt(OPTS["adam"]), push, mask,
+                        order, info)
+    assert info.cpu().tolist() == info_1.cpu().tolist() and info_1.cpu().tolist()[1] == 0
+    assert torch.equal(order, order_1) and torch.equal(mask, mask_1)
+    assert torch.equal(theta, theta_1) and torch.equal(s[0], s1[0]) and torch.equal(s[1], s1[1])
+    assert all(torch.equal(copies[r], theta_1) for r in range(R))
