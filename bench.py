@@ -286,9 +286,16 @@ N_STATE = {"sgd": 0, "momentum": 1, "rmsprop": 2, "adam": 2, "adagrad": 1}
 N_SETS = 16  # arrival/tag draws rotate, so the kept set differs from step to step
 
 
+def it(i: int) -> int:
+    """The iteration number a step passes to the library: 0, 1, 0, 1, ...  Consecutive iterations differ in
+    parity, as the iterations of a real server do (the kernels walk through the columns in alternating directions),
+    and draw i % N_SETS carries the tags of iteration it(i) (N_SETS is even)."""
+    return i & 1
+
+
 def selection_sets(cfg, dev):
     arr = [torch.from_numpy(wl.arrivals(cfg.seed, t, cfg.W)).to(dev) for t in range(N_SETS)]
-    tag = [torch.from_numpy(wl.tags(cfg.seed, t, cfg.W, cfg.N) - t).to(dev) for t in range(N_SETS)]  # relative to t = 0
+    tag = [torch.from_numpy(wl.tags(cfg.seed, t, cfg.W, cfg.N) - t + it(t)).to(dev) for t in range(N_SETS)]
     return arr, tag
 
 
@@ -367,22 +374,22 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
         group_order = torch.zeros(n_machines, dtype=torch.int32, device=dev)
         order = torch.zeros(W, dtype=torch.int32, device=dev)
         info = torch.zeros(3, dtype=torch.int32, device=dev)
-        tag_d = [torch.zeros(W, dtype=torch.int32, device=dev)] * N_SETS  # every worker current: all machines count
+        tag_d = [torch.full((W,), it(k), dtype=torch.int32, device=dev) for k in range(N_SETS)]  # every worker current
         kept_mean = n_machines * W / machines  # exact when the machines are equally large
 
     def step(i):
         opt.step = i + 1
         if machines:
-            sgdb.sgdb_step_grouped(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], group, 0, machines, n_machines, theta, s0,
+            sgdb.sgdb_step_grouped(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], group, it(i), machines, n_machines, theta, s0,
                                    s1, opt, mask, group_order, order, info)
         elif deadline is not None:
-            sgdb.sgdb_step_deadline(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, deadline, 1, theta, s0, s1, opt,
+            sgdb.sgdb_step_deadline(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], it(i), deadline, 1, theta, s0, s1, opt,
                                     mask, order, info)
         elif ema:  # the step plus the running average of the parameters (last line of the server's loop)
-            sgdb.sgdb_step_ema(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, avg, 0.9999,
+            sgdb.sgdb_step_ema(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], it(i), N, b, theta, s0, s1, opt, avg, 0.9999,
                                mask, order, info)
         else:
-            sgdb.sgdb_step(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, mask, order, info)
+            sgdb.sgdb_step(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], it(i), N, b, theta, s0, s1, opt, mask, order, info)
 
     def check():
         assert info.cpu().tolist()[1] == 0, "a step reported a device-side error"
@@ -419,7 +426,7 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
 
         def separate_step(i):
             opt.step = i + 1
-            sgdb.sgdb_select(arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, mask, order, info)
+            sgdb.sgdb_select(arr_d[i % N_SETS], tag_d[i % N_SETS], it(i), N, b, mask, order, info)
             sgdb.sgdb_aggregate(grad, P, N, order, info, mean)
             sgdb.sgdb_update(theta, s0, s1, mean, opt, info)
 
@@ -438,7 +445,7 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
 
         def ema_step(i):
             opt.step = i + 1
-            sgdb.sgdb_step_ema(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, avg_v, 0.9999,
+            sgdb.sgdb_step_ema(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], it(i), N, b, theta, s0, s1, opt, avg_v, 0.9999,
                                mask, order, info)
 
         ms = time_steps(ema_step, 20, 3)
@@ -451,7 +458,7 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
 
         def deadline_step(i):
             opt.step = i + 1
-            sgdb.sgdb_step_deadline(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, dl, 1, theta, s0, s1, opt, mask,
+            sgdb.sgdb_step_deadline(grad, P, arr_d[i % N_SETS], tag_d[i % N_SETS], it(i), dl, 1, theta, s0, s1, opt, mask,
                                     order_w, info)
 
         ms = time_steps(deadline_step, 20 - 20 % N_SETS + N_SETS, 3)  # whole rotations of the draws: the kept count varies
@@ -462,11 +469,11 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
             group = torch.from_numpy((np.arange(W) // 4).astype(np.int32)).to(dev)
             group_order = torch.zeros(m_kept, dtype=torch.int32, device=dev)
             info3 = torch.zeros(3, dtype=torch.int32, device=dev)
-            current = torch.zeros(W, dtype=torch.int32, device=dev)
+            current = [torch.full((W,), par, dtype=torch.int32, device=dev) for par in (0, 1)]
 
             def grouped_step(i):
                 opt.step = i + 1
-                sgdb.sgdb_step_grouped(grad, P, arr_d[i % N_SETS], current, group, 0, m_all, m_kept, theta, s0, s1, opt,
+                sgdb.sgdb_step_grouped(grad, P, arr_d[i % N_SETS], current[it(i)], group, it(i), m_all, m_kept, theta, s0, s1, opt,
                                        mask, group_order, order_w, info3)
 
             ms = time_steps(grouped_step, 20, 3)
@@ -480,7 +487,7 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
 
         def rows_step(i):
             opt.step = i + 1
-            sgdb.sgdb_step_rows(rows_all, grad.dtype, P, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt, None,
+            sgdb.sgdb_step_rows(rows_all, grad.dtype, P, arr_d[i % N_SETS], tag_d[i % N_SETS], it(i), N, b, theta, s0, s1, opt, None,
                                 mask, order, info)
 
         ms = time_steps(rows_step, 20, 3)
@@ -499,7 +506,7 @@ def setup_flat(cfg, dev, sgdb, seed, ema=False, deadline=None, machines=0):
             def servers_step(i):
                 opt.step = i + 1
                 for j, (first, n) in enumerate(ranges):
-                    sgdb.sgdb_step_rows(row_tables[j], grad.dtype, n, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b,
+                    sgdb.sgdb_step_rows(row_tables[j], grad.dtype, n, arr_d[i % N_SETS], tag_d[i % N_SETS], it(i), N, b,
                                         cut(copies[j], first, n), cut(s0, first, n), cut(s1, first, n), opt, push_tables[j],
                                         mask, order, info)
 
@@ -583,13 +590,13 @@ def setup_segmented(cfg, dev, sgdb, seed):
 
     def step(i):
         opt.step = i + 1
-        sgdb.sgdb_step_segmented(table, len(segs), segs[0][3].dtype, arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b,
+        sgdb.sgdb_step_segmented(table, len(segs), segs[0][3].dtype, arr_d[i % N_SETS], tag_d[i % N_SETS], it(i), N, b,
                                  opt, mask, order, info)
 
     def per_tensor_step(i):
         opt.step = i + 1
         for theta, s0, s1, grad in segs:
-            sgdb.sgdb_step(grad, theta.numel(), arr_d[i % N_SETS], tag_d[i % N_SETS], 0, N, b, theta, s0, s1, opt,
+            sgdb.sgdb_step(grad, theta.numel(), arr_d[i % N_SETS], tag_d[i % N_SETS], it(i), N, b, theta, s0, s1, opt,
                            mask, order, info, ld=grad.stride(0))
 
     def check():
@@ -652,11 +659,11 @@ def setup_arrivals(cfg, dev, sgdb, seed):
         # the batched fused step on the same rows, for comparison
         mask, order, finfo = selection_outputs(N + 4, N, dev)
         arr = torch.from_numpy(wl.arrivals(cfg.seed + 4, 0, N + 4)).to(dev)
-        tag = torch.zeros(N + 4, dtype=torch.int32, device=dev)
+        tag = [torch.full((N + 4,), par, dtype=torch.int32, device=dev) for par in (0, 1)]
 
         def batched(i):
             opt.step = i + 1
-            sgdb.sgdb_step(grad[: N + 4], P, arr, tag, 0, N, 4, theta, s0, s1, opt, mask, order, finfo)
+            sgdb.sgdb_step(grad[: N + 4], P, arr, tag[it(i)], it(i), N, 4, theta, s0, s1, opt, mask, order, finfo)
 
         ms = time_steps(batched, 10, 3)
         return {"b_sweep": out, "bytes_per_accepted_arrival": P * 12, "batched_fused_step_ms": ms,
@@ -795,11 +802,11 @@ def run_native(args, cfg):
         h_order = torch.empty(N, dtype=torch.int32, pin_memory=True)
         h_info = torch.empty(2, dtype=torch.int32, pin_memory=True)
         h_arr = [torch.from_numpy(wl.arrivals(cfg.seed, t, W)).pin_memory() for t in range(N_SETS)]
-        h_tag = [torch.from_numpy(wl.tags(cfg.seed, t, W, N) - t).pin_memory() for t in range(N_SETS)]
+        h_tag = [torch.from_numpy(wl.tags(cfg.seed, t, W, N) - t + it(t)).pin_memory() for t in range(N_SETS)]
 
         def host_step(i):
             opt.step = i + 1
-            status = sgdb.sgdb_step_host(h_grad, P, h_arr[i % N_SETS], h_tag[i % N_SETS], 0, N, b, theta, s0, s1, opt,
+            status = sgdb.sgdb_step_host(h_grad, P, h_arr[i % N_SETS], h_tag[i % N_SETS], it(i), N, b, theta, s0, s1, opt,
                                          h_theta, h_mask, h_order, h_info, ws)
             assert status == 0
 

@@ -278,6 +278,7 @@ void set_in_kernel_selection(StreamParams* p, const float* d_arrival, const int3
   p->arrival = d_arrival;
   p->tags = d_tags;
   p->t = t;
+  p->reverse = t & 1;  // consecutive iterations walk through the columns in opposite directions
   p->W = W;
   p->deadline = kNoDeadline;
   p->keep_all = false;
@@ -880,6 +881,7 @@ sgdb_status_t sgdb_step_host(const void* h_grad, sgdb_dtype_t dt, int64_t P, int
     p.order = d_order;
     p.info = d_info;
     p.status_out = d_info + 1;
+    p.reverse = t & 1;
     p.h = h;
     st = launch_stream(dt, ep, p, s);
     if (st != SGDB_OK) return st;
