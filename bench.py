@@ -47,9 +47,10 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0  # earlier measurement on this machine, used only when MEASURED_PEAKS.json is absent
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM traffic of one fused-step launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
-# as bytes per algorithmic byte; valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"src_digest": "d3cf9f22412bc48f", "dram_bytes_per_algorithmic_byte": 0.9946}
+# DRAM traffic of one full-size fused-step launch in steady state from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum, caches left alone), as bytes per algorithmic byte; valid only for the kernel sources whose
+# digest is recorded with it.
+NCU_TRAFFIC = {"src_digest": "26cc691490d24e95", "dram_bytes_per_algorithmic_byte": 0.9891}
 
 
 def kernel_source_digest() -> str:
@@ -883,7 +884,7 @@ def run_servers(args, cfg):
     arr_d, tag_d = selection_sets(cfg, dev)
 
     def step(i):
-        srv.step(0, arr_d[i % N_SETS], tag_d[i % N_SETS], update=i + 1)
+        srv.step(it(i), arr_d[i % N_SETS], tag_d[i % N_SETS], update=i + 1)
 
     def barrier():
         if world > 1:
